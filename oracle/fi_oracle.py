@@ -1,0 +1,184 @@
+"""ctypes front end of the fp64 CPU oracle (`fi_oracle.c`) plus the cascade driver.
+
+TEST INFRASTRUCTURE ONLY.  Imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg; never by the product path.  Shares no code with
+the CUDA path.  See the header of `fi_oracle.c` for what is computed and which
+passages of the paper each step follows.
+
+`cascade()` follows Pseudocode 1 (FreezeInference): stage l looks up only the
+requests that no earlier stage froze; a hit records (label, confidence, stage);
+requests that survive every stage keep label -1 and exit_stage = number of
+stages, standing for "the model's own output layer answers".
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "fi_oracle.c")
+_LIB = os.path.join(_HERE, "libfi_oracle.so")
+
+METRIC_SQL2, METRIC_L2 = 0, 1
+RULE_CONF_GT, RULE_DIST_LE = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain -O2 plus OpenMP; no fast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-ftree-vectorize", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        vp, i64, i32, dbl = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_double
+        _lib.fio_sqdist.argtypes = [vp, vp, i32, i64, i64, i64, vp]
+        _lib.fio_sqdist.restype = None
+        _lib.fio_select.argtypes = [vp, i64, i32, vp, vp]
+        _lib.fio_select.restype = None
+        _lib.fio_vote.argtypes = [vp, vp, vp, i32, i32, i32, dbl, vp, vp, vp]
+        _lib.fio_vote.restype = None
+        _lib.fio_lookup.argtypes = [vp, i64, vp, i64, vp, vp, vp, i32, i64, i64, i32, i32, i32, dbl,
+                                    vp, vp, vp, vp, vp, vp]
+        _lib.fio_lookup.restype = None
+        _lib.fio_compact.argtypes = [vp, vp, i64, vp]
+        _lib.fio_compact.restype = i64
+    return _lib
+
+
+def set_threads(n: int) -> None:
+    """Number of OpenMP threads the next calls use (1 = the paper's single-thread prototype, Sec. 5)."""
+    rt = ctypes.CDLL("libgomp.so.1")
+    rt.omp_set_num_threads(int(n))
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _dtype_code(a: np.ndarray) -> int:
+    if a.dtype == np.float32:
+        return 0
+    if a.dtype == np.uint16:
+        return 1
+    raise TypeError("vectors must be float32 or uint16 (bf16 bit patterns)")
+
+
+def sqdist(queries: np.ndarray, cache: np.ndarray) -> np.ndarray:
+    """D[b][n] = sum_j (q_bj - c_nj)^2 in fp64."""
+    q = np.ascontiguousarray(queries)
+    x = np.ascontiguousarray(cache)
+    assert q.dtype == x.dtype and q.shape[1] == x.shape[1]
+    D = np.empty((q.shape[0], x.shape[0]), dtype=np.float64)
+    _load().fio_sqdist(_ptr(q), _ptr(x), _dtype_code(x), q.shape[0], x.shape[0], x.shape[1], _ptr(D))
+    return D
+
+
+def select(D_row: np.ndarray, kk: int):
+    """The kk smallest of one distance row under the order (D, n)."""
+    D_row = np.ascontiguousarray(D_row, dtype=np.float64)
+    kk = min(kk, D_row.shape[0])
+    od = np.empty(max(kk, 1), dtype=np.float64)
+    oi = np.empty(max(kk, 1), dtype=np.int64)
+    if kk > 0:
+        _load().fio_select(_ptr(D_row), D_row.shape[0], kk, _ptr(od), _ptr(oi))
+    return od[:kk], oi[:kk]
+
+
+def vote(nd: Sequence[float], nlabel: Sequence[int], nweight: Optional[Sequence[float]] = None, *,
+         metric: int = METRIC_SQL2, rule: int = RULE_CONF_GT, tau: float = 0.0):
+    """Label, confidence and hit from neighbour tuples given in ascending (distance, index) order."""
+    nd = np.ascontiguousarray(nd, dtype=np.float64)
+    nl = np.ascontiguousarray(nlabel, dtype=np.int32)
+    nw = np.ones_like(nd) if nweight is None else np.ascontiguousarray(nweight, dtype=np.float64)
+    label = ctypes.c_int32(0)
+    conf = ctypes.c_double(0.0)
+    hit = ctypes.c_uint8(0)
+    _load().fio_vote(_ptr(nd), _ptr(nl), _ptr(nw), len(nd), metric, rule, float(tau),
+                     ctypes.byref(label), ctypes.byref(conf), ctypes.byref(hit))
+    return int(label.value), float(conf.value), bool(hit.value)
+
+
+@dataclass
+class LookupResult:
+    label: np.ndarray      # [B] int32
+    conf: np.ndarray       # [B] float64
+    hit: np.ndarray        # [B] uint8
+    nd: np.ndarray         # [B, k] float64 squared distances, ascending, +inf padded
+    ni: np.ndarray         # [B, k] int64 cache indices, -1 padded
+    next_d: np.ndarray     # [B] float64 squared distance of the (k+1)-th neighbour, +inf if none
+
+
+def lookup(queries: np.ndarray, cache: np.ndarray, labels: np.ndarray, *, k: int, tau: float,
+           rule: int = RULE_CONF_GT, metric: int = METRIC_SQL2, weights: Optional[np.ndarray] = None,
+           row_idx: Optional[np.ndarray] = None) -> LookupResult:
+    q = np.ascontiguousarray(queries)
+    x = np.ascontiguousarray(cache)
+    lab = np.ascontiguousarray(labels, dtype=np.int32)
+    w = None if weights is None else np.ascontiguousarray(weights, dtype=np.float32)
+    ridx = None if row_idx is None else np.ascontiguousarray(row_idx, dtype=np.int32)
+    assert q.dtype == x.dtype and q.ndim == 2 and x.ndim == 2
+    n, dim = x.shape
+    assert q.shape[1] == dim and lab.shape[0] == n
+    batch = q.shape[0] if ridx is None else ridx.shape[0]
+    res = LookupResult(np.empty(batch, np.int32), np.empty(batch, np.float64), np.empty(batch, np.uint8),
+                       np.empty((batch, k), np.float64), np.empty((batch, k), np.int64), np.empty(batch, np.float64))
+    _load().fio_lookup(_ptr(q), q.shape[1], _ptr(ridx), batch, _ptr(x), _ptr(lab), _ptr(w), _dtype_code(x), n, dim,
+                       int(k), int(metric), int(rule), float(tau), _ptr(res.label), _ptr(res.conf), _ptr(res.hit),
+                       _ptr(res.nd), _ptr(res.ni), _ptr(res.next_d))
+    return res
+
+
+def compact(active: np.ndarray, hit: np.ndarray) -> np.ndarray:
+    """Ids of `active` whose look-up missed, order kept (Sec. 5, batch reconstruction)."""
+    a = np.ascontiguousarray(active, dtype=np.int32)
+    h = np.ascontiguousarray(hit, dtype=np.uint8)
+    out = np.empty(max(1, a.shape[0]), dtype=np.int32)
+    m = _load().fio_compact(_ptr(a), _ptr(h), a.shape[0], _ptr(out))
+    return out[:m].copy()
+
+
+@dataclass
+class CascadeResult:
+    final_label: np.ndarray    # [B0] int32, -1 = never frozen
+    final_conf: np.ndarray     # [B0] float64
+    exit_stage: np.ndarray     # [B0] int32, number of stages = never frozen
+    active: List[np.ndarray]   # active[l] = request ids that reached stage l (ascending); one extra entry = survivors
+    stage_results: List[LookupResult]
+
+
+def cascade(stage_queries: Sequence[np.ndarray], stage_caches: Sequence[np.ndarray],
+            stage_labels: Sequence[np.ndarray], taus: Sequence[float], *, k: int, rule: int = RULE_CONF_GT,
+            metric: int = METRIC_SQL2, stage_weights: Optional[Sequence[Optional[np.ndarray]]] = None) -> CascadeResult:
+    n_stage = len(stage_caches)
+    b0 = stage_queries[0].shape[0]
+    final_label = np.full(b0, -1, np.int32)
+    final_conf = np.zeros(b0, np.float64)
+    exit_stage = np.full(b0, n_stage, np.int32)
+    active = [np.arange(b0, dtype=np.int32)]
+    results = []
+    for l in range(n_stage):
+        ids = active[-1]
+        w = None if stage_weights is None else stage_weights[l]
+        r = lookup(stage_queries[l], stage_caches[l], stage_labels[l], k=k, tau=taus[l], rule=rule, metric=metric,
+                   weights=w, row_idx=ids)
+        frozen = r.hit.astype(bool)
+        final_label[ids[frozen]] = r.label[frozen]
+        final_conf[ids[frozen]] = r.conf[frozen]
+        exit_stage[ids[frozen]] = l
+        results.append(r)
+        active.append(compact(ids, r.hit))
+    return CascadeResult(final_label, final_conf, exit_stage, active, results)
