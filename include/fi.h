@@ -1,0 +1,191 @@
+/*
+ * fi.h — C ABI of the per-layer approximate cache of Freeze Inference (arXiv 2002.02645).
+ *
+ * One `fi_cache_t` is the cache of one DNN layer (Pseudocode 1: CACHE[layer], THRESHOLDS[layer]).
+ * The online operations are the cache look-up API of Sec. 3 on a batch of requests and the
+ * per-layer cascade step of Pseudocode 1 (FreezeInference) with the batch reconstruction that
+ * Sec. 5 asks for.  All device work runs in CUDA kernels built for sm_100a; there is no CPU path.
+ *
+ * Conventions
+ *   - Unless a parameter says "host", every data pointer is a DEVICE pointer on the cache's device,
+ *     allocated and owned by the caller.  The library owns only what `fi_cache_create` allocates
+ *     (rows, labels, weights, squared norms, scratch) and frees it in `fi_cache_destroy`.
+ *   - `cuda_stream` is a `cudaStream_t` passed as `void*` (NULL = the legacy default stream).  Calls
+ *     enqueue work on it and return without synchronising, except where stated.
+ *   - Calls that use the same cache share its scratch memory and must be ordered on one stream
+ *     (or otherwise serialised); different caches are independent.
+ *   - Every failure is a returned status; nothing aborts, throws, or traps on the device.  A wait
+ *     inside a kernel that runs out (bounded) sets a device status word, which `fi_cache_poll_status`
+ *     reads.  `fi_last_error` gives a text for the last failure on the calling thread.
+ *   - Vectors are row-major with contiguous elements: float32 (FI_F32) or bfloat16 (FI_BF16).
+ *     Queries have the dtype of the cache.  bfloat16 rows must start on 16-byte boundaries
+ *     (base pointer 16-byte aligned, leading dimension a multiple of 8 elements), and
+ *     dim must be a multiple of 8 (bf16) or 4 (f32).
+ */
+#ifndef FI_H_
+#define FI_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fi_cache fi_cache_t; /* opaque; one per layer */
+
+typedef enum {
+    FI_OK = 0,
+    FI_ERR_INVALID_ARG = 1,
+    FI_ERR_CAPACITY = 2,
+    FI_ERR_OOM = 3,
+    FI_ERR_CUDA = 4,
+    FI_ERR_UNSUPPORTED = 5,
+    FI_ERR_TIMEOUT = 6
+} fi_status_t;
+
+typedef enum { FI_F32 = 0, FI_BF16 = 1 } fi_dtype_t;
+
+/* Hit rule.  FI_HIT_CONF_GT is the paper's: hit iff confidence > threshold, strict (Pseudocode 1,
+ * FreezeInference; Sec. 2.1 "exceeds").  FI_HIT_DIST_LE: hit iff the smallest distance among the
+ * neighbours that carry the winning label is <= threshold (for k = 1: nearest-neighbour distance). */
+typedef enum { FI_HIT_CONF_GT = 0, FI_HIT_DIST_LE = 1 } fi_hit_rule_t;
+
+/* The d_j of the confidence sum (Sec. 3): squared L2 distance, or its square root. */
+typedef enum { FI_METRIC_SQL2 = 0, FI_METRIC_L2 = 1 } fi_metric_t;
+
+/* Which kernels serve a look-up.  AUTO: the streaming kernel for batches of at most 4 and for float32
+ * caches, the tensor-core distance GEMM otherwise.  The other two force a path (bf16 only for GEMM). */
+typedef enum { FI_PATH_AUTO = 0, FI_PATH_STREAM = 1, FI_PATH_GEMM = 2 } fi_path_t;
+
+typedef struct {
+    int32_t dim;         /* vector length d */
+    int32_t dtype;       /* fi_dtype_t */
+    int64_t capacity;    /* maximum number of entries */
+    int32_t num_classes; /* labels must lie in [0, num_classes) */
+    int32_t k;           /* neighbours per look-up, 1..32 */
+    int32_t rule;        /* fi_hit_rule_t */
+    int32_t metric;      /* fi_metric_t */
+    float threshold;     /* THRESHOLDS[layer] */
+    int32_t device;      /* CUDA device ordinal */
+    int32_t max_batch;   /* largest batch a look-up on this cache may carry (sizes the scratch) */
+    int32_t path;        /* fi_path_t */
+} fi_cache_config_t;
+
+/* Results of a look-up, one entry per batch slot i (the i-th request of the batch). */
+typedef struct {
+    int32_t *label;      /* [batch] predicted label, -1 for an empty cache */
+    float *conf;         /* [batch] confidence C of that label (+inf when a neighbour is at distance 0) */
+    uint8_t *hit;        /* [batch] 1 = frozen here */
+    float *topk_dist;    /* [batch*k] nullable; squared L2 distances of the k neighbours, ascending, +inf padded */
+    int32_t *topk_idx;   /* [batch*k] nullable; their cache indices, -1 padded */
+} fi_lookup_out_t;
+
+/* State of a batch walking through the layers.  Request ids are 0..batch0-1. */
+typedef struct {
+    const int32_t *active_idx;   /* in : ids alive at this stage, ascending; NULL = all of 0..batch0-1 */
+    const int32_t *active_count; /* in : how many; NULL = batch0 */
+    int32_t *miss_idx;           /* out: ids alive at the next stage, ascending; [batch0] */
+    int32_t *miss_count;         /* out: how many; [1] */
+    int32_t *final_label;        /* [batch0] written for the requests frozen at this stage */
+    int32_t *exit_stage;         /* [batch0] written with `stage` for them */
+    float *final_conf;           /* [batch0] written with their confidence */
+    int32_t stage;               /* index of this stage */
+    int32_t batch0;              /* size of the original batch */
+} fi_cascade_state_t;
+
+/*
+ * Create the (empty) cache of one layer: CACHE[layer] = {} and THRESHOLDS[layer] of Pseudocode 1.
+ * Allocates capacity*dim elements plus labels, weights, norms and look-up scratch on cfg->device.
+ * Synchronous.  Errors: INVALID_ARG (null, dim/k/capacity/max_batch out of range, dim not a multiple
+ * of 8 (bf16) or 4 (f32)), OOM, CUDA.  On error *out is NULL.
+ */
+fi_status_t fi_cache_create(const fi_cache_config_t *cfg, fi_cache_t **out);
+
+/* Free everything the cache owns.  Synchronises the device.  NULL is accepted. */
+fi_status_t fi_cache_destroy(fi_cache_t *cache);
+
+/*
+ * Append n entries <vector, label[, weight]>: ConstructCache of Pseudocode 1 appends <IO[item][layer],
+ * Y[item]>; with `weights` an entry is the k-means form of Sec. 4, <cluster centre, majority label,
+ * fraction of the majority label>.  vecs: [n x dim] device, row-major, contiguous rows; labels: [n] device
+ * int32; weights: [n] device float or NULL (= 1.0).  Also computes each row's squared norm.  Asynchronous
+ * on the stream; label values are not range-checked on the host (they are opaque to the look-up).
+ * Errors: CAPACITY when size + n > capacity (nothing is written), INVALID_ARG, CUDA.
+ */
+fi_status_t fi_cache_insert(fi_cache_t *cache, const void *vecs, const int32_t *labels, const float *weights,
+                            int64_t n, void *cuda_stream);
+
+/* Set THRESHOLDS[layer] (Pseudocode 1; Sec. 3.1 (ii) describes how the offline phase picks it). */
+fi_status_t fi_cache_set_threshold(fi_cache_t *cache, float tau);
+
+/* Choose the kernels later look-ups use (fi_path_t).  UNSUPPORTED for FI_PATH_GEMM on a float32 cache. */
+fi_status_t fi_cache_set_path(fi_cache_t *cache, int32_t path);
+
+/* Number of entries currently stored. */
+int64_t fi_cache_size(const fi_cache_t *cache);
+
+/*
+ * The cache look-up API of Sec. 3 for a batch: for each request the k nearest cached entries under squared
+ * L2 (ties by smaller index), per label i among them S_i = m_i/k and C_i = S_i * sum_j w_j/d_j, the label
+ * with the largest C_i and that C_i, and the hit flag under the cache's rule and threshold.  With
+ * fewer than k entries, k_eff = min(k, size) replaces k.
+ *   queries          [rows x ld_elems] device; request i is row row_idx[i] (or row i when row_idx is NULL)
+ *   ld_elems         leading dimension in elements (>= dim)
+ *   row_idx          [batch_max] device int32 or NULL
+ *   batch_max        upper bound of the batch, 0..max_batch; sizes the launch
+ *   batch_count_dev  [1] device int32 holding the actual batch (<= batch_max), or NULL = batch_max; read
+ *                    by the kernels, never by the host, so a cascade needs no host round trip
+ *   out              device arrays; slots >= the actual batch are left untouched
+ * Asynchronous.  Errors: INVALID_ARG, UNSUPPORTED, CUDA.
+ */
+fi_status_t fi_cache_lookup_batch(const fi_cache_t *cache, const void *queries, int64_t ld_elems,
+                                  const int32_t *row_idx, int32_t batch_max, const int32_t *batch_count_dev,
+                                  const fi_lookup_out_t *out, void *cuda_stream);
+
+/* Start a cascade: final_label = -1, final_conf = 0, exit_stage = num_stages for all batch0 requests
+ * (the value a request keeps when no layer freezes it: the model's output layer answers, Pseudocode 1). */
+fi_status_t fi_cascade_init(const fi_cascade_state_t *state, int32_t num_stages, int32_t device, void *cuda_stream);
+
+/*
+ * One layer of FreezeInference (Pseudocode 1) for a whole batch: look up the activations of the requests
+ * still alive in this layer's cache; a hit freezes the request (its label, confidence and stage are
+ * recorded); the misses are compacted, order kept, into the batch of the next layer (Sec. 5, "reconstruct
+ * the batch after each layer to remove the items that have been frozen").
+ *   stage_acts  [batch0 x ld_elems] device: row r = activation of request r at this layer
+ * Needs state->batch0 <= max_batch of the cache.  Asynchronous; the count stays on the device.
+ */
+fi_status_t fi_cascade_step(const fi_cache_t *stage_cache, const void *stage_acts, int64_t ld_elems,
+                            const fi_cascade_state_t *state, void *cuda_stream);
+
+/*
+ * End-to-end variants with HOST buffers: copy the inputs to the device, run the same kernels, copy the
+ * results back, and synchronise the stream before returning.
+ * fi_cache_lookup_batch_host: queries [batch x dim] host, contiguous; out arrays are host pointers.
+ * fi_cascade_run_host: acts[l] = [batch0 x dim_l] host activations of every request at stage l; runs
+ * fi_cascade_init and num_stages steps; outputs [batch0] host arrays; stage_arrivals [num_stages+1] host,
+ * nullable: number of requests that reached each stage, last entry = never frozen.
+ */
+fi_status_t fi_cache_lookup_batch_host(const fi_cache_t *cache, const void *queries_host, int32_t batch,
+                                       const fi_lookup_out_t *out_host, void *cuda_stream);
+fi_status_t fi_cascade_run_host(fi_cache_t *const *stage_caches, int32_t num_stages, const void *const *acts_host,
+                                int32_t batch0, int32_t *final_label_host, int32_t *exit_stage_host,
+                                float *final_conf_host, int32_t *stage_arrivals_host, void *cuda_stream);
+
+/* Synchronise the device and return FI_ERR_TIMEOUT if a kernel of this cache gave up on a bounded wait
+ * since the last poll (the word is cleared), FI_OK otherwise. */
+fi_status_t fi_cache_poll_status(fi_cache_t *cache);
+
+/* Number of kernels this library has launched in the calling process (all caches). */
+int64_t fi_launch_count(void);
+
+/* Text of the last error on the calling thread ("" if none).  The pointer stays valid until the next call
+ * of the library on this thread. */
+const char *fi_last_error(void);
+
+/* Name of a status code. */
+const char *fi_status_string(fi_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FI_H_ */

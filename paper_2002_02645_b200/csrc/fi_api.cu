@@ -1,0 +1,559 @@
+// The C ABI declared in include/fi.h: argument checks, memory ownership, and the order in which the
+// kernels of a look-up / cascade step are enqueued.  No arithmetic of the method lives here.
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "fi_internal.cuh"
+
+namespace fi {
+
+namespace {
+thread_local char g_err[512] = "";
+std::atomic<long long> g_launches{0};
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        if (prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+fi_status_t cuda_fail(cudaError_t e, const char *what) {
+    set_error("%s: %s", what, cudaGetErrorString(e));
+    cudaGetLastError();
+    return e == cudaErrorMemoryAllocation ? FI_ERR_OOM : FI_ERR_CUDA;
+}
+
+__global__ void fill_f32_kernel(float *p, int64_t n, float v) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) p[i] = v;
+}
+
+template <typename T>
+fi_status_t dev_alloc(T **p, size_t count, const char *what) {
+    *p = nullptr;
+    if (count == 0) count = 1;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(p), count * sizeof(T));
+    if (e != cudaSuccess) return cuda_fail(e, what);
+    return FI_OK;
+}
+
+void free_all(fi_cache *c) {
+    cudaFree(c->rows);
+    cudaFree(c->labels);
+    cudaFree(c->weights);
+    cudaFree(c->norms);
+    cudaFree(c->part_score);
+    cudaFree(c->part_idx);
+    cudaFree(c->q_compact);
+    cudaFree(c->slot_label);
+    cudaFree(c->slot_conf);
+    cudaFree(c->slot_hit);
+    cudaFree(c->plan_dev);
+    cudaFree(c->status_dev);
+    cudaFree(c->h2d_stage);
+    cudaFree(c->casc_buf);
+}
+
+int resolve_path(const fi_cache *c, int batch_max) {
+    if (c->size == 0) return FI_PATH_STREAM;   // nothing to contract with; the streaming kernel reports "no neighbour"
+    if (c->cfg.path == FI_PATH_STREAM || c->cfg.path == FI_PATH_GEMM) return c->cfg.path;
+    if (c->cfg.dtype == FI_F32 || batch_max <= kStreamMaxBatch) return FI_PATH_STREAM;
+    return FI_PATH_GEMM;
+}
+
+fi_status_t ensure_part_scratch(fi_cache *c, size_t entries) {
+    if (entries <= c->part_entries) return FI_OK;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e, "synchronising before growing the look-up scratch");
+    cudaFree(c->part_score);
+    cudaFree(c->part_idx);
+    c->part_score = nullptr;
+    c->part_idx = nullptr;
+    c->part_entries = 0;
+    fi_status_t st = dev_alloc(&c->part_score, entries, "allocating candidate scores");
+    if (st != FI_OK) return st;
+    st = dev_alloc(&c->part_idx, entries, "allocating candidate indices");
+    if (st != FI_OK) return st;
+    c->part_entries = entries;
+    return FI_OK;
+}
+
+fi_status_t lookup_impl(fi_cache *c, const void *queries, int64_t ld, const int32_t *row_idx, int32_t batch_max,
+                        const int32_t *count_dev, const fi_lookup_out_t &out, cudaStream_t stream) {
+    if (batch_max == 0) return FI_OK;
+    const int path = resolve_path(c, batch_max);
+    FinalizeArgs fa;
+    fa.queries = queries;
+    fa.ld_elems = ld;
+    fa.row_idx = row_idx;
+    fa.batch_max = batch_max;
+    fa.count_dev = count_dev;
+    fa.out = out;
+    fi_status_t st;
+    if (path == FI_PATH_STREAM) {
+        int parts = 1;
+        st = launch_stream_lookup(c, queries, ld, row_idx, batch_max, count_dev, &parts, stream);
+        if (st != FI_OK) return st;
+        fa.parts = parts;
+        fa.list_len = c->cfg.k;
+        fa.refine = 0;
+    } else {
+        if (c->cfg.dtype != FI_BF16) {
+            set_error("the tensor-core path needs a bf16 cache");
+            return FI_ERR_UNSUPPORTED;
+        }
+        st = ensure_part_scratch(c, gemm_part_entries(batch_max, c->size, c->sm_count, c->cfg.k));
+        if (st != FI_OK) return st;
+        const void *qsrc = queries;
+        int64_t qld = ld;
+        if (row_idx) {
+            st = launch_gather_rows(queries, ld, row_idx, batch_max, count_dev, c->q_compact, c->cfg.dim, c->elem_size, stream);
+            if (st != FI_OK) return st;
+            qsrc = c->q_compact;
+            qld = c->cfg.dim;
+            fa.queries = qsrc;
+            fa.ld_elems = qld;
+            fa.row_idx = nullptr;
+        }
+        st = launch_gemm_select(c, qsrc, qld, batch_max, count_dev, stream);
+        if (st != FI_OK) return st;
+        fa.parts = -1;
+        fa.list_len = -1;
+        fa.refine = 1;
+    }
+    return launch_finalize(c, fa, stream);
+}
+
+}  // namespace
+
+void set_error(const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+}
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+fi_status_t check_launch(const char *what) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, what);
+    return FI_OK;
+}
+
+}  // namespace fi
+
+using namespace fi;
+
+extern "C" {
+
+fi_status_t fi_cache_create(const fi_cache_config_t *cfg, fi_cache_t **out) {
+    if (out) *out = nullptr;
+    if (!cfg || !out) {
+        set_error("fi_cache_create: null argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    const bool bf16 = cfg->dtype == FI_BF16;
+    if ((cfg->dtype != FI_F32 && !bf16) || cfg->dim <= 0 || cfg->dim % (bf16 ? 8 : 4) != 0 || cfg->capacity <= 0 ||
+        cfg->k < 1 || cfg->k > kMaxK || cfg->max_batch < 1 || cfg->num_classes < 1 ||
+        (cfg->rule != FI_HIT_CONF_GT && cfg->rule != FI_HIT_DIST_LE) ||
+        (cfg->metric != FI_METRIC_SQL2 && cfg->metric != FI_METRIC_L2) || cfg->path < FI_PATH_AUTO ||
+        cfg->path > FI_PATH_GEMM) {
+        set_error("fi_cache_create: invalid configuration (dim %d dtype %d capacity %lld k %d max_batch %d)", cfg->dim,
+                  cfg->dtype, (long long)cfg->capacity, cfg->k, cfg->max_batch);
+        return FI_ERR_INVALID_ARG;
+    }
+    if (cfg->path == FI_PATH_GEMM && !bf16) {
+        set_error("fi_cache_create: the tensor-core path needs a bf16 cache");
+        return FI_ERR_UNSUPPORTED;
+    }
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device < 0 || cfg->device >= ndev) {
+        cudaGetLastError();
+        set_error("fi_cache_create: no CUDA device %d", cfg->device);
+        return FI_ERR_CUDA;
+    }
+    DeviceGuard guard(cfg->device);
+    if (!guard.ok) {
+        set_error("fi_cache_create: cannot select device %d", cfg->device);
+        return FI_ERR_CUDA;
+    }
+    fi_cache *c = new (std::nothrow) fi_cache();
+    if (!c) {
+        set_error("fi_cache_create: out of host memory");
+        return FI_ERR_OOM;
+    }
+    memset(c, 0, sizeof *c);
+    c->cfg = *cfg;
+    c->elem_size = bf16 ? 2 : 4;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) {
+        delete c;
+        return cuda_fail(cudaGetLastError(), "fi_cache_create: device properties");
+    }
+    c->sm_count = prop.multiProcessorCount;
+
+    fi_status_t st = FI_OK;
+    auto need = [&](fi_status_t s) {
+        if (st == FI_OK) st = s;
+    };
+    unsigned char *rows = nullptr;
+    need(dev_alloc(&rows, (size_t)cfg->capacity * cfg->dim * c->elem_size, "allocating cache rows"));
+    c->rows = rows;
+    if (st == FI_OK) need(dev_alloc(&c->labels, (size_t)cfg->capacity, "allocating labels"));
+    if (st == FI_OK) need(dev_alloc(&c->weights, (size_t)cfg->capacity, "allocating weights"));
+    if (st == FI_OK) need(dev_alloc(&c->norms, (size_t)cfg->capacity, "allocating norms"));
+    // candidate lists: the streaming kernel cuts the rows into up to 16 ranges per SM for a group of 4 queries
+    size_t entries = (size_t)16 * c->sm_count * 4 * cfg->k;
+    if (entries < (size_t)cfg->max_batch * cfg->k * 2) entries = (size_t)cfg->max_batch * cfg->k * 2;
+    if (bf16) {
+        size_t g = gemm_part_entries(cfg->max_batch, cfg->capacity, c->sm_count, cfg->k);
+        if (g > entries) entries = g;
+    }
+    if (st == FI_OK) need(dev_alloc(&c->part_score, entries, "allocating candidate scores"));
+    if (st == FI_OK) need(dev_alloc(&c->part_idx, entries, "allocating candidate indices"));
+    c->part_entries = entries;
+    if (st == FI_OK && bf16) {
+        unsigned char *qc = nullptr;
+        need(dev_alloc(&qc, (size_t)cfg->max_batch * cfg->dim * c->elem_size, "allocating the gathered-query buffer"));
+        c->q_compact = qc;
+    }
+    if (st == FI_OK) need(dev_alloc(&c->slot_label, (size_t)cfg->max_batch, "allocating slot labels"));
+    if (st == FI_OK) need(dev_alloc(&c->slot_conf, (size_t)cfg->max_batch, "allocating slot confidences"));
+    if (st == FI_OK) need(dev_alloc(&c->slot_hit, (size_t)cfg->max_batch, "allocating slot hit flags"));
+    if (st == FI_OK) need(dev_alloc(&c->plan_dev, 1, "allocating the plan"));
+    if (st == FI_OK) need(dev_alloc(&c->status_dev, 1, "allocating the status word"));
+    if (st == FI_OK) {
+        cudaError_t e = cudaMemset(c->status_dev, 0, sizeof(int32_t));
+        if (e != cudaSuccess) st = cuda_fail(e, "clearing the status word");
+    }
+    if (st != FI_OK) {
+        free_all(c);
+        delete c;
+        return st;
+    }
+    *out = c;
+    return FI_OK;
+}
+
+fi_status_t fi_cache_destroy(fi_cache_t *c) {
+    if (!c) return FI_OK;
+    DeviceGuard guard(c->cfg.device);
+    cudaDeviceSynchronize();
+    free_all(c);
+    cudaGetLastError();
+    delete c;
+    return FI_OK;
+}
+
+fi_status_t fi_cache_insert(fi_cache_t *c, const void *vecs, const int32_t *labels, const float *weights, int64_t n,
+                            void *cuda_stream) {
+    if (!c || n < 0 || (n > 0 && (!vecs || !labels))) {
+        set_error("fi_cache_insert: null or negative argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    if (n == 0) return FI_OK;
+    if (c->size + n > c->cfg.capacity) {
+        set_error("fi_cache_insert: %lld entries do not fit (size %lld, capacity %lld)", (long long)n, (long long)c->size,
+                  (long long)c->cfg.capacity);
+        return FI_ERR_CAPACITY;
+    }
+    if ((reinterpret_cast<uintptr_t>(vecs) & 15) != 0) {
+        set_error("fi_cache_insert: vectors must be 16-byte aligned");
+        return FI_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(c->cfg.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t row_bytes = (size_t)c->cfg.dim * c->elem_size;
+    unsigned char *dst = static_cast<unsigned char *>(c->rows) + (size_t)c->size * row_bytes;
+    cudaError_t e = cudaMemcpyAsync(dst, vecs, (size_t)n * row_bytes, cudaMemcpyDeviceToDevice, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cache_insert: copying rows");
+    e = cudaMemcpyAsync(c->labels + c->size, labels, (size_t)n * sizeof(int32_t), cudaMemcpyDeviceToDevice, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cache_insert: copying labels");
+    if (weights) {
+        e = cudaMemcpyAsync(c->weights + c->size, weights, (size_t)n * sizeof(float), cudaMemcpyDeviceToDevice, stream);
+        if (e != cudaSuccess) return cuda_fail(e, "fi_cache_insert: copying weights");
+    } else {
+        int grid = (int)((n + 255) / 256 < 1024 ? (n + 255) / 256 : 1024);
+        fill_f32_kernel<<<grid, 256, 0, stream>>>(c->weights + c->size, n, 1.0f);
+        count_launch();
+        fi_status_t st = check_launch("fill_f32_kernel");
+        if (st != FI_OK) return st;
+    }
+    fi_status_t st = launch_row_norms(dst, c->cfg.dtype, n, c->cfg.dim, c->norms + c->size, stream);
+    if (st != FI_OK) return st;
+    c->size += n;
+    c->tmaps_ready = false;
+    return FI_OK;
+}
+
+fi_status_t fi_cache_set_threshold(fi_cache_t *c, float tau) {
+    if (!c) {
+        set_error("fi_cache_set_threshold: null cache");
+        return FI_ERR_INVALID_ARG;
+    }
+    c->cfg.threshold = tau;
+    return FI_OK;
+}
+
+fi_status_t fi_cache_set_path(fi_cache_t *c, int32_t path) {
+    if (!c || path < FI_PATH_AUTO || path > FI_PATH_GEMM) {
+        set_error("fi_cache_set_path: invalid argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    if (path == FI_PATH_GEMM && c->cfg.dtype != FI_BF16) {
+        set_error("fi_cache_set_path: the tensor-core path needs a bf16 cache");
+        return FI_ERR_UNSUPPORTED;
+    }
+    c->cfg.path = path;
+    return FI_OK;
+}
+
+int64_t fi_cache_size(const fi_cache_t *c) { return c ? c->size : 0; }
+
+fi_status_t fi_cache_lookup_batch(const fi_cache_t *cache, const void *queries, int64_t ld_elems, const int32_t *row_idx,
+                                  int32_t batch_max, const int32_t *batch_count_dev, const fi_lookup_out_t *out,
+                                  void *cuda_stream) {
+    if (!cache || !out || batch_max < 0 || (batch_max > 0 && (!queries || !out->label || !out->conf || !out->hit))) {
+        set_error("fi_cache_lookup_batch: null or negative argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    if (batch_max > cache->cfg.max_batch) {
+        set_error("fi_cache_lookup_batch: batch %d exceeds max_batch %d", batch_max, cache->cfg.max_batch);
+        return FI_ERR_INVALID_ARG;
+    }
+    const int align_elems = 16 / (int)cache->elem_size;
+    if (ld_elems < cache->cfg.dim || ld_elems % align_elems != 0 || (reinterpret_cast<uintptr_t>(queries) & 15) != 0) {
+        set_error("fi_cache_lookup_batch: rows must start on 16-byte boundaries (ld %lld, dim %d)", (long long)ld_elems,
+                  cache->cfg.dim);
+        return FI_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(cache->cfg.device);
+    // the handle is const for the caller: the look-up does not change the cache's contents, only its scratch
+    return lookup_impl(const_cast<fi_cache *>(cache), queries, ld_elems, row_idx, batch_max, batch_count_dev, *out,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+fi_status_t fi_cascade_init(const fi_cascade_state_t *state, int32_t num_stages, int32_t device, void *cuda_stream) {
+    if (!state || state->batch0 < 0 || num_stages < 0 ||
+        (state->batch0 > 0 && (!state->final_label || !state->exit_stage || !state->final_conf))) {
+        set_error("fi_cascade_init: null or negative argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(device);
+    return launch_cascade_init(*state, num_stages, static_cast<cudaStream_t>(cuda_stream));
+}
+
+fi_status_t fi_cascade_step(const fi_cache_t *cache, const void *stage_acts, int64_t ld_elems,
+                            const fi_cascade_state_t *state, void *cuda_stream) {
+    if (!cache || !state || state->batch0 < 0 || !state->miss_idx || !state->miss_count ||
+        (state->batch0 > 0 && (!stage_acts || !state->final_label || !state->exit_stage || !state->final_conf))) {
+        set_error("fi_cascade_step: null or negative argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    if (state->batch0 > cache->cfg.max_batch) {
+        set_error("fi_cascade_step: batch %d exceeds max_batch %d", state->batch0, cache->cfg.max_batch);
+        return FI_ERR_INVALID_ARG;
+    }
+    if (state->miss_idx == state->active_idx) {
+        set_error("fi_cascade_step: miss_idx must not alias active_idx");
+        return FI_ERR_INVALID_ARG;
+    }
+    fi_cache *c = const_cast<fi_cache *>(cache);
+    fi_lookup_out_t out;
+    out.label = c->slot_label;
+    out.conf = c->slot_conf;
+    out.hit = c->slot_hit;
+    out.topk_dist = nullptr;
+    out.topk_idx = nullptr;
+    fi_status_t st = fi_cache_lookup_batch(cache, stage_acts, ld_elems, state->active_idx, state->batch0,
+                                           state->active_count, &out, cuda_stream);
+    if (st != FI_OK) return st;
+    DeviceGuard guard(cache->cfg.device);
+    return launch_compact(c, *state, static_cast<cudaStream_t>(cuda_stream));
+}
+
+fi_status_t fi_cache_lookup_batch_host(const fi_cache_t *cache, const void *queries_host, int32_t batch,
+                                       const fi_lookup_out_t *out_host, void *cuda_stream) {
+    if (!cache || !out_host || batch < 0 ||
+        (batch > 0 && (!queries_host || !out_host->label || !out_host->conf || !out_host->hit))) {
+        set_error("fi_cache_lookup_batch_host: null or negative argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    if (batch > cache->cfg.max_batch) {
+        set_error("fi_cache_lookup_batch_host: batch %d exceeds max_batch %d", batch, cache->cfg.max_batch);
+        return FI_ERR_INVALID_ARG;
+    }
+    if (batch == 0) return FI_OK;
+    fi_cache *c = const_cast<fi_cache *>(cache);
+    DeviceGuard guard(c->cfg.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int k = c->cfg.k;
+    const size_t q_bytes = (size_t)batch * c->cfg.dim * c->elem_size;
+    const size_t q_pad = (q_bytes + 255) & ~(size_t)255;
+    const size_t out_bytes = (size_t)batch * (4 + 4 + 4 + 8 * (size_t)k);   // hit padded to 4 bytes per slot
+    const size_t need = q_pad + out_bytes + 256;
+    if (need > c->h2d_stage_bytes) {
+        cudaError_t e = cudaDeviceSynchronize();
+        if (e != cudaSuccess) return cuda_fail(e, "fi_cache_lookup_batch_host: synchronising");
+        cudaFree(c->h2d_stage);
+        c->h2d_stage = nullptr;
+        c->h2d_stage_bytes = 0;
+        e = cudaMalloc(&c->h2d_stage, need);
+        if (e != cudaSuccess) return cuda_fail(e, "fi_cache_lookup_batch_host: allocating staging");
+        c->h2d_stage_bytes = need;
+    }
+    unsigned char *base = static_cast<unsigned char *>(c->h2d_stage);
+    fi_lookup_out_t dev;
+    dev.label = reinterpret_cast<int32_t *>(base + q_pad);
+    dev.conf = reinterpret_cast<float *>(base + q_pad + (size_t)batch * 4);
+    dev.topk_dist = reinterpret_cast<float *>(base + q_pad + (size_t)batch * 8);
+    dev.topk_idx = reinterpret_cast<int32_t *>(base + q_pad + (size_t)batch * 8 + (size_t)batch * k * 4);
+    dev.hit = base + q_pad + (size_t)batch * 8 + (size_t)batch * k * 8;
+    cudaError_t e = cudaMemcpyAsync(base, queries_host, q_bytes, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cache_lookup_batch_host: copying queries");
+    fi_status_t st = lookup_impl(c, base, c->cfg.dim, nullptr, batch, nullptr, dev, stream);
+    if (st != FI_OK) return st;
+    e = cudaMemcpyAsync(out_host->label, dev.label, (size_t)batch * 4, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out_host->conf, dev.conf, (size_t)batch * 4, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out_host->hit, dev.hit, (size_t)batch, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess && out_host->topk_dist)
+        e = cudaMemcpyAsync(out_host->topk_dist, dev.topk_dist, (size_t)batch * k * 4, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess && out_host->topk_idx)
+        e = cudaMemcpyAsync(out_host->topk_idx, dev.topk_idx, (size_t)batch * k * 4, cudaMemcpyDeviceToHost, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cache_lookup_batch_host: copying results");
+    e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cache_lookup_batch_host: synchronising");
+    return FI_OK;
+}
+
+fi_status_t fi_cascade_run_host(fi_cache_t *const *caches, int32_t num_stages, const void *const *acts_host,
+                                int32_t batch0, int32_t *final_label_host, int32_t *exit_stage_host,
+                                float *final_conf_host, int32_t *stage_arrivals_host, void *cuda_stream) {
+    if (!caches || !acts_host || num_stages < 1 || batch0 < 0 || !final_label_host || !exit_stage_host || !final_conf_host) {
+        set_error("fi_cascade_run_host: null or negative argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    for (int l = 0; l < num_stages; ++l) {
+        if (!caches[l] || !acts_host[l] || caches[l]->cfg.device != caches[0]->cfg.device || batch0 > caches[l]->cfg.max_batch) {
+            set_error("fi_cascade_run_host: stage %d: null cache or activations, other device, or batch above max_batch", l);
+            return FI_ERR_INVALID_ARG;
+        }
+    }
+    if (batch0 == 0) return FI_OK;
+    fi_cache *c0 = caches[0];
+    DeviceGuard guard(c0->cfg.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // device staging: activations of every stage, then the cascade state
+    size_t act_off[64];
+    if (num_stages > 63) {
+        set_error("fi_cascade_run_host: at most 63 stages");
+        return FI_ERR_INVALID_ARG;
+    }
+    size_t total = 0;
+    for (int l = 0; l < num_stages; ++l) {
+        act_off[l] = total;
+        total += ((size_t)batch0 * caches[l]->cfg.dim * caches[l]->elem_size + 255) & ~(size_t)255;
+    }
+    const size_t state_off = total;
+    const size_t nb = (size_t)batch0;
+    total += (5 * nb + (size_t)num_stages + 8) * 4 + 256;
+    if (total > c0->h2d_stage_bytes) {
+        cudaError_t e = cudaDeviceSynchronize();
+        if (e != cudaSuccess) return cuda_fail(e, "fi_cascade_run_host: synchronising");
+        cudaFree(c0->h2d_stage);
+        c0->h2d_stage = nullptr;
+        c0->h2d_stage_bytes = 0;
+        e = cudaMalloc(&c0->h2d_stage, total);
+        if (e != cudaSuccess) return cuda_fail(e, "fi_cascade_run_host: allocating staging");
+        c0->h2d_stage_bytes = total;
+    }
+    unsigned char *base = static_cast<unsigned char *>(c0->h2d_stage);
+    int32_t *ibase = reinterpret_cast<int32_t *>(base + state_off);
+    int32_t *idx[2] = {ibase, ibase + nb};
+    int32_t *final_label = ibase + 2 * nb;
+    int32_t *exit_stage = ibase + 3 * nb;
+    float *final_conf = reinterpret_cast<float *>(ibase + 4 * nb);
+    int32_t *counts = ibase + 5 * nb;   // counts[l] = arrivals at stage l; counts[0] unused (= batch0)
+
+    cudaError_t e = cudaSuccess;
+    for (int l = 0; l < num_stages && e == cudaSuccess; ++l)
+        e = cudaMemcpyAsync(base + act_off[l], acts_host[l], (size_t)batch0 * caches[l]->cfg.dim * caches[l]->elem_size,
+                            cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cascade_run_host: copying activations");
+
+    fi_cascade_state_t st;
+    memset(&st, 0, sizeof st);
+    st.batch0 = batch0;
+    st.final_label = final_label;
+    st.exit_stage = exit_stage;
+    st.final_conf = final_conf;
+    fi_status_t rc = fi_cascade_init(&st, num_stages, c0->cfg.device, cuda_stream);
+    if (rc != FI_OK) return rc;
+    for (int l = 0; l < num_stages; ++l) {
+        st.stage = l;
+        st.active_idx = l == 0 ? nullptr : idx[(l - 1) & 1];
+        st.active_count = l == 0 ? nullptr : counts + l;
+        st.miss_idx = idx[l & 1];
+        st.miss_count = counts + l + 1;
+        rc = fi_cascade_step(caches[l], base + act_off[l], caches[l]->cfg.dim, &st, cuda_stream);
+        if (rc != FI_OK) return rc;
+    }
+    e = cudaMemcpyAsync(final_label_host, final_label, nb * 4, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(exit_stage_host, exit_stage, nb * 4, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(final_conf_host, final_conf, nb * 4, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess && stage_arrivals_host && num_stages > 0)
+        e = cudaMemcpyAsync(stage_arrivals_host + 1, counts + 1, (size_t)num_stages * 4, cudaMemcpyDeviceToHost, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cascade_run_host: copying results");
+    e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cascade_run_host: synchronising");
+    if (stage_arrivals_host) stage_arrivals_host[0] = batch0;
+    return FI_OK;
+}
+
+fi_status_t fi_cache_poll_status(fi_cache_t *c) {
+    if (!c) {
+        set_error("fi_cache_poll_status: null cache");
+        return FI_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(c->cfg.device);
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cache_poll_status: synchronising");
+    int32_t word = 0;
+    e = cudaMemcpy(&word, c->status_dev, sizeof word, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cache_poll_status: reading the status word");
+    if (word != 0) {
+        cudaMemset(c->status_dev, 0, sizeof word);
+        set_error("a kernel gave up on a bounded wait (code %d, site %d)", word & 0xFF, word >> 8);
+        return FI_ERR_TIMEOUT;
+    }
+    return FI_OK;
+}
+
+int64_t fi_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
+
+const char *fi_last_error(void) { return g_err; }
+
+const char *fi_status_string(fi_status_t s) {
+    switch (s) {
+        case FI_OK: return "FI_OK";
+        case FI_ERR_INVALID_ARG: return "FI_ERR_INVALID_ARG";
+        case FI_ERR_CAPACITY: return "FI_ERR_CAPACITY";
+        case FI_ERR_OOM: return "FI_ERR_OOM";
+        case FI_ERR_CUDA: return "FI_ERR_CUDA";
+        case FI_ERR_UNSUPPORTED: return "FI_ERR_UNSUPPORTED";
+        case FI_ERR_TIMEOUT: return "FI_ERR_TIMEOUT";
+    }
+    return "FI_?";
+}
+
+}  // extern "C"

@@ -1,0 +1,355 @@
+// Per-query finish of a look-up and the batch reconstruction.
+//
+// finalize_kernel (one CTA per query): merge the candidate lists that the distance kernels left per range of
+// cache rows, optionally recompute the exact squared distance sum_j (q_j - c_j)^2 of each candidate in fp32
+// (the GEMM's ||q||^2 + ||c||^2 - 2 q.c form cancels badly for close pairs), order by (distance, index), then
+// apply the confidence heuristic of Sec. 3 (S_i = m_i/k, C_i = S_i * sum_j w_j/d_j, arg-max) and the hit rule of
+// Pseudocode 1.
+//
+// compact_kernel (one CTA): warp-ballot stream compaction of the misses, order kept (Sec. 5, rebuilding the
+// batch after each layer), and the scatter of (label, confidence, stage) for the requests frozen here.
+#include "fi_internal.cuh"
+
+namespace fi {
+
+namespace {
+
+constexpr int kFinThreads = 256;
+constexpr int kFinWarps = kFinThreads / 32;
+
+struct FinalizeParams {
+    const void *X;
+    const int32_t *labels;
+    const float *weights;
+    int64_t n_entries;
+    int dim;
+    const void *Q;
+    int64_t ldq;
+    const int32_t *row_idx;
+    int32_t batch_max;
+    const int32_t *count_dev;
+    const float *part_score;
+    const int32_t *part_idx;
+    int parts;
+    int list_len;
+    const GemmPlan *plan;
+    int refine;
+    int k;
+    int metric;
+    int rule;
+    float tau;
+    int32_t *out_label;
+    float *out_conf;
+    uint8_t *out_hit;
+    float *out_topk_dist;
+    int32_t *out_topk_idx;
+};
+
+__device__ __forceinline__ uint4 ld16(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+template <typename T>
+__device__ __forceinline__ float sqdiff16(uint4 q, uint4 x, float acc);
+template <>
+__device__ __forceinline__ float sqdiff16<float>(uint4 q, uint4 x, float acc) {
+    float d0 = __uint_as_float(q.x) - __uint_as_float(x.x);
+    float d1 = __uint_as_float(q.y) - __uint_as_float(x.y);
+    float d2 = __uint_as_float(q.z) - __uint_as_float(x.z);
+    float d3 = __uint_as_float(q.w) - __uint_as_float(x.w);
+    acc = fmaf(d0, d0, acc);
+    acc = fmaf(d1, d1, acc);
+    acc = fmaf(d2, d2, acc);
+    return fmaf(d3, d3, acc);
+}
+template <>
+__device__ __forceinline__ float sqdiff16<uint16_t>(uint4 q, uint4 x, float acc) {
+    uint32_t qw[4] = {q.x, q.y, q.z, q.w};
+    uint32_t xw[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float d0 = __uint_as_float(qw[i] << 16) - __uint_as_float(xw[i] << 16);
+        float d1 = __uint_as_float(qw[i] & 0xFFFF0000u) - __uint_as_float(xw[i] & 0xFFFF0000u);
+        acc = fmaf(d0, d0, acc);
+        acc = fmaf(d1, d1, acc);
+    }
+    return acc;
+}
+
+__device__ __forceinline__ bool pair_less(float s, int i, float t, int j) { return s < t || (s == t && i < j); }
+
+template <typename T>
+__global__ void __launch_bounds__(kFinThreads) finalize_kernel(FinalizeParams p) {
+    __shared__ float cand_s[kMaxK];
+    __shared__ float cand_d[kMaxK];
+    __shared__ int32_t cand_i[kMaxK];
+    __shared__ float red_s[kFinWarps];
+    __shared__ int32_t red_i[kFinWarps];
+    __shared__ int32_t s_cand_n;
+
+    const int count = p.count_dev ? min(*p.count_dev, p.batch_max) : p.batch_max;
+    const int b = blockIdx.x;
+    if (b >= count) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int parts = p.plan ? p.plan->parts : p.parts;
+    const int list_len = p.plan ? p.plan->list_len : p.list_len;
+    const int entries = parts * list_len;
+    const float *ps = p.part_score + (int64_t)b * entries;
+    const int32_t *pi = p.part_idx + (int64_t)b * entries;
+    int want = p.refine ? list_len : p.k;
+    if (want > kMaxK) want = kMaxK;
+    const float kInf = __int_as_float(0x7F800000);
+
+    // ---- merge: repeatedly take the smallest (score, index) pair above the previous pick
+    float prev_s = -kInf;
+    int prev_i = -1;
+    int cand_n = 0;
+    for (int r = 0; r < want; ++r) {
+        float best_s = kInf;
+        int best_i = 0x7FFFFFFF;
+        for (int e = tid; e < entries; e += kFinThreads) {
+            float s = ps[e];
+            int i = pi[e];
+            if (i < 0) continue;
+            bool above = r == 0 || pair_less(prev_s, prev_i, s, i);
+            if (above && pair_less(s, i, best_s, best_i)) {
+                best_s = s;
+                best_i = i;
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            float os = __shfl_xor_sync(0xFFFFFFFFu, best_s, o);
+            int oi = __shfl_xor_sync(0xFFFFFFFFu, best_i, o);
+            if (pair_less(os, oi, best_s, best_i)) {
+                best_s = os;
+                best_i = oi;
+            }
+        }
+        if (lane == 0) {
+            red_s[warp] = best_s;
+            red_i[warp] = best_i;
+        }
+        __syncthreads();
+        best_s = red_s[0];
+        best_i = red_i[0];
+#pragma unroll
+        for (int w = 1; w < kFinWarps; ++w)
+            if (pair_less(red_s[w], red_i[w], best_s, best_i)) {
+                best_s = red_s[w];
+                best_i = red_i[w];
+            }
+        __syncthreads();
+        if (best_i == 0x7FFFFFFF) break;   // lists exhausted
+        if (tid == 0) {
+            cand_s[r] = best_s;
+            cand_i[r] = best_i;
+        }
+        prev_s = best_s;
+        prev_i = best_i;
+        cand_n = r + 1;
+    }
+    __syncthreads();
+
+    // ---- exact distances of the candidates
+    if (p.refine) {
+        const int64_t qr = p.row_idx ? (int64_t)p.row_idx[b] : (int64_t)b;
+        const T *q = reinterpret_cast<const T *>(p.Q) + qr * p.ldq;
+        const int chunks = p.dim / (16 / (int)sizeof(T));
+        for (int j = warp; j < cand_n; j += kFinWarps) {
+            const T *x = reinterpret_cast<const T *>(p.X) + (int64_t)cand_i[j] * p.dim;
+            float a0 = 0.f, a1 = 0.f;
+            int c = lane;
+            for (; c + 32 < chunks; c += 64) {
+                uint4 x0 = ld16(reinterpret_cast<const uint4 *>(x) + c);
+                uint4 x1 = ld16(reinterpret_cast<const uint4 *>(x) + c + 32);
+                uint4 q0 = ld16(reinterpret_cast<const uint4 *>(q) + c);
+                uint4 q1 = ld16(reinterpret_cast<const uint4 *>(q) + c + 32);
+                a0 = sqdiff16<T>(q0, x0, a0);
+                a1 = sqdiff16<T>(q1, x1, a1);
+            }
+            for (; c < chunks; c += 32)
+                a0 = sqdiff16<T>(ld16(reinterpret_cast<const uint4 *>(q) + c), ld16(reinterpret_cast<const uint4 *>(x) + c), a0);
+            float a = a0 + a1;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
+            if (lane == 0) cand_d[j] = a;
+        }
+    } else {
+        if (tid < cand_n) cand_d[tid] = cand_s[tid];
+    }
+    __syncthreads();
+
+    // ---- order by (distance, index), vote, hit
+    if (tid == 0) {
+        for (int a = 1; a < cand_n; ++a) {
+            float d = cand_d[a];
+            int i = cand_i[a];
+            int pos = a;
+            while (pos > 0 && pair_less(d, i, cand_d[pos - 1], cand_i[pos - 1])) {
+                cand_d[pos] = cand_d[pos - 1];
+                cand_i[pos] = cand_i[pos - 1];
+                --pos;
+            }
+            cand_d[pos] = d;
+            cand_i[pos] = i;
+        }
+        const int k_eff = cand_n < p.k ? cand_n : p.k;
+        int32_t lab[kMaxK];
+        float wgt[kMaxK];
+        for (int j = 0; j < k_eff; ++j) {
+            lab[j] = p.labels[cand_i[j]];
+            wgt[j] = p.weights[cand_i[j]];
+        }
+        int32_t best_label = -1;
+        float best_c = 0.f, best_dwin = 0.f;
+        int best_m = 0;
+        for (int a = 0; a < k_eff; ++a) {
+            bool seen = false;
+            for (int e = 0; e < a; ++e) seen |= (lab[e] == lab[a]);
+            if (seen) continue;   // scored at its nearest occurrence
+            int m = 0;
+            float sum = 0.f;
+            for (int j = a; j < k_eff; ++j) {
+                if (lab[j] != lab[a]) continue;
+                float dj = p.metric == FI_METRIC_L2 ? sqrtf(cand_d[j]) : cand_d[j];
+                sum += wgt[j] / dj;
+                ++m;
+            }
+            float c = ((float)m / (float)k_eff) * sum;
+            if (best_label < 0 || c > best_c || (c == best_c && m > best_m)) {
+                best_label = lab[a];
+                best_c = c;
+                best_m = m;
+                best_dwin = p.metric == FI_METRIC_L2 ? sqrtf(cand_d[a]) : cand_d[a];
+            }
+        }
+        bool hit = k_eff > 0 && (p.rule == FI_HIT_CONF_GT ? best_c > p.tau : best_dwin <= p.tau);
+        p.out_label[b] = best_label;
+        p.out_conf[b] = best_c;
+        p.out_hit[b] = hit ? 1 : 0;
+        if (p.out_topk_dist)
+            for (int j = 0; j < p.k; ++j) p.out_topk_dist[(int64_t)b * p.k + j] = j < k_eff ? cand_d[j] : kInf;
+        if (p.out_topk_idx)
+            for (int j = 0; j < p.k; ++j) p.out_topk_idx[(int64_t)b * p.k + j] = j < k_eff ? cand_i[j] : -1;
+    }
+}
+
+// ---------------------------------------------------------------- K4: miss compaction
+__global__ void __launch_bounds__(1024)
+compact_kernel(const int32_t *__restrict__ active_idx, const int32_t *__restrict__ active_count, int32_t batch0,
+               const int32_t *__restrict__ slot_label, const float *__restrict__ slot_conf,
+               const uint8_t *__restrict__ slot_hit, int32_t stage, int32_t *__restrict__ miss_idx,
+               int32_t *__restrict__ miss_count, int32_t *__restrict__ final_label, int32_t *__restrict__ exit_stage,
+               float *__restrict__ final_conf) {
+    __shared__ int32_t warp_total[32];
+    __shared__ int32_t warp_base[32];
+    __shared__ int32_t running;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int count = active_count ? min(*active_count, batch0) : batch0;
+    if (tid == 0) running = 0;
+    __syncthreads();
+    for (int base = 0; base < count; base += 1024) {
+        const int i = base + tid;
+        const bool valid = i < count;
+        int32_t id = 0;
+        bool miss = false;
+        if (valid) {
+            id = active_idx ? active_idx[i] : i;
+            miss = slot_hit[i] == 0;
+            if (!miss) {
+                final_label[id] = slot_label[i];
+                final_conf[id] = slot_conf[i];
+                exit_stage[id] = stage;
+            }
+        }
+        const unsigned ballot = __ballot_sync(0xFFFFFFFFu, miss);
+        const int before = __popc(ballot & ((1u << lane) - 1u));
+        if (lane == 0) warp_total[warp] = __popc(ballot);
+        __syncthreads();
+        if (warp == 0) {
+            int t = warp_total[lane];
+            int incl = t;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            warp_base[lane] = running + incl - t;
+            __syncwarp();
+            if (lane == 31) running += incl;
+        }
+        __syncthreads();
+        if (miss) miss_idx[warp_base[warp] + before] = id;
+        __syncthreads();
+    }
+    if (tid == 0) *miss_count = running;
+}
+
+__global__ void cascade_init_kernel(int32_t batch0, int32_t num_stages, int32_t *final_label, int32_t *exit_stage,
+                                    float *final_conf) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < batch0; i += gridDim.x * blockDim.x) {
+        final_label[i] = -1;
+        exit_stage[i] = num_stages;
+        final_conf[i] = 0.f;
+    }
+}
+
+}  // namespace
+
+fi_status_t launch_finalize(const fi_cache *c, const FinalizeArgs &a, cudaStream_t stream) {
+    if (a.batch_max <= 0) return FI_OK;
+    FinalizeParams p;
+    p.X = c->rows;
+    p.labels = c->labels;
+    p.weights = c->weights;
+    p.n_entries = c->size;
+    p.dim = c->cfg.dim;
+    p.Q = a.queries;
+    p.ldq = a.ld_elems;
+    p.row_idx = a.row_idx;
+    p.batch_max = a.batch_max;
+    p.count_dev = a.count_dev;
+    p.part_score = c->part_score;
+    p.part_idx = c->part_idx;
+    p.parts = a.parts;
+    p.list_len = a.list_len;
+    p.plan = a.parts < 0 ? c->plan_dev : nullptr;
+    p.refine = a.refine;
+    p.k = c->cfg.k;
+    p.metric = c->cfg.metric;
+    p.rule = c->cfg.rule;
+    p.tau = c->cfg.threshold;
+    p.out_label = a.out.label;
+    p.out_conf = a.out.conf;
+    p.out_hit = a.out.hit;
+    p.out_topk_dist = a.out.topk_dist;
+    p.out_topk_idx = a.out.topk_idx;
+    if (c->cfg.dtype == FI_F32)
+        finalize_kernel<float><<<a.batch_max, kFinThreads, 0, stream>>>(p);
+    else
+        finalize_kernel<uint16_t><<<a.batch_max, kFinThreads, 0, stream>>>(p);
+    count_launch();
+    return check_launch("finalize_kernel");
+}
+
+fi_status_t launch_compact(const fi_cache *c, const fi_cascade_state_t &st, cudaStream_t stream) {
+    compact_kernel<<<1, 1024, 0, stream>>>(st.active_idx, st.active_count, st.batch0, c->slot_label, c->slot_conf,
+                                           c->slot_hit, st.stage, st.miss_idx, st.miss_count, st.final_label,
+                                           st.exit_stage, st.final_conf);
+    count_launch();
+    return check_launch("compact_kernel");
+}
+
+fi_status_t launch_cascade_init(const fi_cascade_state_t &st, int32_t num_stages, cudaStream_t stream) {
+    if (st.batch0 <= 0) return FI_OK;
+    int grid = (st.batch0 + 255) / 256;
+    if (grid > 1024) grid = 1024;
+    cascade_init_kernel<<<grid, 256, 0, stream>>>(st.batch0, num_stages, st.final_label, st.exit_stage, st.final_conf);
+    count_launch();
+    return check_launch("cascade_init_kernel");
+}
+
+}  // namespace fi

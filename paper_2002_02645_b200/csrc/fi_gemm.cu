@@ -1,0 +1,503 @@
+// Distance GEMM with fused per-row select for bf16 caches (sm_100a: TMA + tcgen05 + TMEM).
+//
+// Neighbour order under ||q - c||^2 = ||q||^2 + ||c||^2 - 2 q.c does not depend on ||q||^2, so the kernel ranks
+// cache rows by the score  s = ||c||^2 - 2 q.c : S = Q X^T is a dense bf16 contraction with fp32 accumulation
+// on the tensor cores; the distance matrix is never written to memory.  Each of the 4 epilogue warps reads
+// accumulator tiles back from TMEM (one query row per thread) and keeps the `list_len` smallest scores of its
+// row in registers.  The exact distances of those few candidates are recomputed afterwards (finalize_kernel).
+//
+// Roles inside a CTA of 192 threads: warp 0 = TMA producer (one lane), warp 1 = TMEM owner and MMA issuer
+// (one lane), warps 2..5 = epilogue.  Shared-memory stages are handed over with mbarriers; the accumulator is
+// double-buffered in TMEM (2 x 256 columns) so the select of one tile overlaps the MMAs of the next.
+// Every wait is bounded: a wait that runs out sets the cache's status word and the CTA drains and returns.
+#include <cuda_bf16.h>
+
+#include "fi_internal.cuh"
+
+namespace fi {
+
+namespace {
+
+constexpr int kBlockK = 64;                       // bf16 elements per k-block: 128 bytes, one swizzle row
+constexpr int kStages = 4;
+constexpr int kMaxTileN = 256;                    // cache rows per tile (MMA N), multiple of 16
+constexpr int kABytes = kTileM * kBlockK * 2;     // 16 KiB
+constexpr int kBBytes = kMaxTileN * kBlockK * 2;  // 32 KiB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kGemmThreads = 192;
+constexpr int kEpiWarps = 4;
+constexpr int kTmemCols = 512;
+constexpr uint64_t kWaitLimitNs = 4000000000ull;  // 4 s: far beyond any tile, short enough to get the GPU back
+
+struct __align__(8) SmemCtl {
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint32_t tmem_base;
+    volatile int32_t abort_flag;
+    GemmPlan plan;
+};
+
+constexpr int kNormSmemBytes = kEpiWarps * 2 * kMaxTileN * 4;   // per epilogue warp, per accumulator buffer
+constexpr int kGemmSmemBytes = 1024 /*alignment slack*/ + kStages * kStageBytes + kNormSmemBytes + (int)sizeof(SmemCtl);
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the abort flag and the status word) when the limit is reached or
+// another thread of the CTA has already given up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, SmemCtl *ctl, int32_t *status, int where) {
+    if (mbar_try(bar, parity)) return true;
+    uint64_t t0 = global_timer_ns();
+    uint32_t spins = 0;
+    while (true) {
+        if (mbar_try(bar, parity)) return true;
+        if ((++spins & 0x3FF) == 0) {
+            if (ctl->abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                ctl->abort_flag = 1;
+                atomicCAS(status, 0, (int32_t)(FI_ERR_TIMEOUT | (where << 8)));
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y)
+        : "memory");
+}
+
+// K-major operand tile in shared memory, rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);   // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                    // leading-dimension offset: unused for swizzled K-major
+    d |= (uint64_t)(1024 >> 4) << 32;          // stride between 8-row groups
+    d |= (uint64_t)1 << 46;                    // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                    // 128-byte swizzle
+    return d;
+}
+// bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n
+__device__ __forceinline__ uint32_t umma_instr_desc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 16 consecutive accumulator columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+// wait for the loads; the registers are listed so that no use of them can move above the wait
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[16]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                   "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15])
+                 :
+                 : "memory");
+}
+
+template <int KP>
+struct TopList {
+    float s[KP];
+    int32_t i[KP];
+    __device__ __forceinline__ void reset() {
+#pragma unroll
+        for (int e = 0; e < KP; ++e) {
+            s[e] = __int_as_float(0x7F800000);
+            i[e] = -1;
+        }
+    }
+    // precondition: sc < s[KP-1].  Equal scores keep their arrival order (smaller index first).
+    __device__ __forceinline__ void insert(float sc, int32_t idx) {
+        s[KP - 1] = sc;
+        i[KP - 1] = idx;
+#pragma unroll
+        for (int e = KP - 1; e > 0; --e) {
+            if (s[e] < s[e - 1]) {
+                float ts = s[e];
+                s[e] = s[e - 1];
+                s[e - 1] = ts;
+                int32_t ti = i[e];
+                i[e] = i[e - 1];
+                i[e - 1] = ti;
+            }
+        }
+    }
+};
+
+struct TileWalk {
+    // cache-row range of this CTA and how it is cut into tiles
+    int col_begin, col_end, tiles, tile_w;
+    __device__ __forceinline__ void setup(const GemmPlan &p, int q, long long n_entries) {
+        long long n_pad = ((n_entries + 15) / 16) * 16;
+        long long b = (long long)q * p.range16 * 16;
+        long long e = b + (long long)p.range16 * 16;
+        if (e > n_pad) e = n_pad;
+        if (b > e) b = e;
+        col_begin = (int)b;
+        col_end = (int)e;
+        int cols = col_end - col_begin;
+        tiles = (cols + kMaxTileN - 1) / kMaxTileN;
+        tile_w = tiles > 0 ? (((cols + tiles - 1) / tiles + 15) / 16) * 16 : 0;
+    }
+    __device__ __forceinline__ int col0(int t) const { return col_begin + t * tile_w; }
+    __device__ __forceinline__ int width(int t) const {
+        int w = col_end - col0(t);
+        return w < tile_w ? w : tile_w;
+    }
+};
+
+template <int KP>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_x64,
+                   const __grid_constant__ CUtensorMap tmap_x16, const float *__restrict__ norms, long long n_entries,
+                   int dim, int batch_max, const int32_t *__restrict__ count_dev, int k,
+                   float *__restrict__ part_score, int32_t *__restrict__ part_idx, GemmPlan *__restrict__ plan_out,
+                   int32_t *__restrict__ status) {
+    extern __shared__ unsigned char smem_raw[];
+    // operand stages need 1024-byte alignment for the 128-byte swizzle
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    unsigned char *stage_base = smem;
+    float *norm_smem = reinterpret_cast<float *>(smem + kStages * kStageBytes);
+    SmemCtl *ctl = reinterpret_cast<SmemCtl *>(smem + kStages * kStageBytes + kNormSmemBytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        int count = count_dev ? min(*count_dev, batch_max) : batch_max;
+        if (count < 0) count = 0;
+        ctl->plan = make_gemm_plan(count, n_entries, (int)gridDim.x, k);
+        ctl->abort_flag = 0;
+        if (blockIdx.x == 0) *plan_out = ctl->plan;
+    }
+    __syncthreads();
+    const GemmPlan plan = ctl->plan;
+    const int m_local = blockIdx.x % plan.mg;
+    const int q = blockIdx.x / plan.mg;
+    if (plan.m_tiles == 0 || plan.range16 == 0 || q >= plan.parts) return;   // whole CTA, before any barrier
+    TileWalk walk;
+    walk.setup(plan, q, n_entries);
+    if (walk.tiles == 0) return;
+    const int num_kb = (dim + kBlockK - 1) / kBlockK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&ctl->tmem_full[a], 1);
+            mbar_init(&ctl->tmem_empty[a], kEpiWarps * 32);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int g = 0; g < plan.groups && ok; ++g) {
+                const int m_tile = g * plan.mg + m_local;
+                if (m_tile >= plan.m_tiles) continue;
+                for (int t = 0; t < walk.tiles && ok; ++t) {
+                    const int col0 = walk.col0(t), w = walk.width(t);
+                    for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                        const int s = it % kStages;
+                        const uint32_t ph = (it / kStages) & 1;
+                        if (!mbar_wait(&ctl->empty[s], ph ^ 1, ctl, status, 1)) {
+                            ok = false;
+                            break;
+                        }
+                        mbar_expect_tx(&ctl->full[s], (uint32_t)(kABytes + w * kBlockK * 2));
+                        const uint32_t a_dst = smem_u32(stage_base + s * kStageBytes);
+                        const uint32_t b_dst = a_dst + kABytes;
+                        tma_load_2d(a_dst, &tmap_q, &ctl->full[s], kb * kBlockK, m_tile * kTileM);
+                        int r = 0;
+                        for (; r + 64 <= w; r += 64)
+                            tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x64, &ctl->full[s], kb * kBlockK, col0 + r);
+                        for (; r < w; r += 16)
+                            tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x16, &ctl->full[s], kb * kBlockK, col0 + r);
+                    }
+                }
+            }
+            if (!ok) {
+                // gave up: let the copies already issued land before the CTA leaves
+                uint32_t issued = it;
+                uint32_t first = issued > (uint32_t)kStages ? issued - kStages : 0;
+                for (uint32_t j = first; j < issued; ++j) {
+                    uint64_t t0 = global_timer_ns();
+                    while (!mbar_try(&ctl->full[j % kStages], (j / kStages) & 1))
+                        if (global_timer_ns() - t0 > 20000000ull) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t it = 0, tile_no = 0;
+            bool ok = true;
+            for (int g = 0; g < plan.groups && ok; ++g) {
+                const int m_tile = g * plan.mg + m_local;
+                if (m_tile >= plan.m_tiles) continue;
+                for (int t = 0; t < walk.tiles && ok; ++t, ++tile_no) {
+                    const int w = walk.width(t);
+                    const uint32_t acc = tile_no & 1, acc_ph = (tile_no >> 1) & 1;
+                    if (!mbar_wait(&ctl->tmem_empty[acc], acc_ph ^ 1, ctl, status, 2)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + acc * kMaxTileN;
+                    const uint32_t idesc = umma_instr_desc(w);
+                    for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                        const int s = it % kStages;
+                        const uint32_t ph = (it / kStages) & 1;
+                        if (!mbar_wait(&ctl->full[s], ph, ctl, status, 3)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t a_addr = smem_u32(stage_base + s * kStageBytes);
+                        const uint64_t adesc = umma_smem_desc(a_addr);
+                        const uint64_t bdesc = umma_smem_desc(a_addr + kABytes);
+#pragma unroll
+                        for (int kk = 0; kk < kBlockK / 16; ++kk)
+                            umma_bf16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | kk) != 0);
+                        umma_commit(&ctl->empty[s]);   // frees the stage once these MMAs have read it
+                    }
+                    if (ok) umma_commit(&ctl->tmem_full[acc]);
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue: per-row select
+        const int ew = warp - 2;              // 0..3, staging slot
+        const int quarter = warp & 3;         // TMEM lanes this warp may read: 32*quarter .. +31
+        const int row_in_tile = quarter * 32 + lane;
+        float *my_norm = norm_smem + ew * (2 * kMaxTileN);
+        TopList<KP> top;
+        uint32_t tile_no = 0;
+        bool ok = true;
+        for (int g = 0; g < plan.groups && ok; ++g) {
+            const int m_tile = g * plan.mg + m_local;
+            if (m_tile >= plan.m_tiles) continue;
+            top.reset();
+            for (int t = 0; t < walk.tiles && ok; ++t, ++tile_no) {
+                const int col0 = walk.col0(t), w = walk.width(t);
+                const uint32_t acc = tile_no & 1, acc_ph = (tile_no >> 1) & 1;
+                float *nrm = my_norm + acc * kMaxTileN;
+                // squared norms of this tile's cache rows; rows past the end get +inf and never enter a list
+                for (int c = lane; c < w; c += 32)
+                    nrm[c] = (long long)(col0 + c) < n_entries ? __ldg(norms + col0 + c) : __int_as_float(0x7F800000);
+                __syncwarp();
+                // the whole warp takes the same decision, so its lanes stay together for the TMEM loads
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, status, 4));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kMaxTileN;
+                for (int c0 = 0; c0 < w; c0 += 16) {
+                    uint32_t v[16];
+                    __syncwarp();
+                    tmem_ld16(taddr + c0, v);
+                    tmem_ld_wait(v);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        float sc = fmaf(-2.f, __uint_as_float(v[j]), nrm[c0 + j]);
+                        if (sc < top.s[KP - 1]) top.insert(sc, col0 + c0 + j);
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(&ctl->tmem_empty[acc]);
+                __syncwarp();
+            }
+            if (ok) {
+                const int row = m_tile * kTileM + row_in_tile;
+                if (row < plan.count) {
+                    const long long o = ((long long)row * plan.parts + q) * KP;
+#pragma unroll
+                    for (int e = 0; e < KP; ++e) {
+                        part_score[o + e] = top.s[e];
+                        part_idx[o + e] = top.i[e];
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 matrix [rows x dim], row pitch ld elements; box = box_rows x 64 elements, 128-byte swizzle, zero fill
+fi_status_t encode_bf16_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t dim, uint64_t ld, uint32_t box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) {
+        set_error("cuTensorMapEncodeTiled is not available from this driver");
+        return FI_ERR_UNSUPPORTED;
+    }
+    cuuint64_t gdim[2] = {dim, rows > 0 ? rows : 1};
+    cuuint64_t gstride[1] = {ld * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kBlockK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled failed with code %d (base %p rows %llu dim %llu ld %llu)", (int)r, base,
+                  (unsigned long long)rows, (unsigned long long)dim, (unsigned long long)ld);
+        return FI_ERR_CUDA;
+    }
+    return FI_OK;
+}
+
+template <int KP>
+fi_status_t launch_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, const int32_t *count_dev, cudaStream_t stream) {
+    static bool attr_set = false;
+    auto kern = gemm_select_kernel<KP>;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) != cudaSuccess) {
+            set_error("cannot reserve %d bytes of shared memory for the distance GEMM", kGemmSmemBytes);
+            cudaGetLastError();
+            return FI_ERR_CUDA;
+        }
+        attr_set = true;
+    }
+    kern<<<c->sm_count, kGemmThreads, kGemmSmemBytes, stream>>>(tq, c->tmap_rows64, c->tmap_rows16, c->norms,
+                                                               (long long)c->size, c->cfg.dim, batch_max, count_dev,
+                                                               c->cfg.k, c->part_score, c->part_idx, c->plan_dev,
+                                                               c->status_dev);
+    count_launch();
+    return check_launch("gemm_select_kernel");
+}
+
+}  // namespace
+
+fi_status_t ensure_tensor_maps(fi_cache *c) {
+    if (c->tmaps_ready) return FI_OK;
+    fi_status_t st = encode_bf16_map(&c->tmap_rows64, c->rows, (uint64_t)c->size, (uint64_t)c->cfg.dim, (uint64_t)c->cfg.dim, 64);
+    if (st != FI_OK) return st;
+    st = encode_bf16_map(&c->tmap_rows16, c->rows, (uint64_t)c->size, (uint64_t)c->cfg.dim, (uint64_t)c->cfg.dim, 16);
+    if (st != FI_OK) return st;
+    c->tmaps_ready = true;
+    return FI_OK;
+}
+
+size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k) {
+    size_t worst = 0;
+    int m_tiles_max = (max_batch + kTileM - 1) / kTileM;
+    for (int mt = 1; mt <= m_tiles_max; ++mt) {
+        GemmPlan p = make_gemm_plan(mt * kTileM, capacity, sm_count, k);
+        size_t e = (size_t)mt * kTileM * (size_t)p.parts * (size_t)p.list_len;
+        if (e > worst) worst = e;
+    }
+    return worst;
+}
+
+fi_status_t launch_gemm_select(fi_cache *c, const void *queries_compact, int64_t ld_elems, int32_t batch_max,
+                               const int32_t *count_dev, cudaStream_t stream) {
+    if (batch_max <= 0) return FI_OK;
+    if (c->size <= 0) {
+        set_error("the distance GEMM needs a non-empty cache");
+        return FI_ERR_INVALID_ARG;
+    }
+    fi_status_t st = ensure_tensor_maps(c);
+    if (st != FI_OK) return st;
+    if ((reinterpret_cast<uintptr_t>(queries_compact) & 15) != 0 || (ld_elems % 8) != 0) {
+        set_error("bf16 queries must be 16-byte aligned with a leading dimension that is a multiple of 8");
+        return FI_ERR_INVALID_ARG;
+    }
+    CUtensorMap tq;
+    st = encode_bf16_map(&tq, queries_compact, (uint64_t)batch_max, (uint64_t)c->cfg.dim, (uint64_t)ld_elems, kTileM);
+    if (st != FI_OK) return st;
+    switch (gemm_list_len(c->cfg.k)) {
+        case 4: return launch_kp<4>(c, tq, batch_max, count_dev, stream);
+        case 8: return launch_kp<8>(c, tq, batch_max, count_dev, stream);
+        case 16: return launch_kp<16>(c, tq, batch_max, count_dev, stream);
+        default: return launch_kp<32>(c, tq, batch_max, count_dev, stream);
+    }
+}
+
+}  // namespace fi

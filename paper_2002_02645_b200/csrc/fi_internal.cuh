@@ -1,0 +1,157 @@
+// Internal declarations shared by the translation units of the library (not part of the ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/fi.h"
+
+namespace fi {
+
+constexpr int kMaxK = 32;          // largest k of a look-up
+constexpr int kStreamMaxBatch = 4; // batches up to this size take the streaming kernel under FI_PATH_AUTO
+constexpr int kTileM = 128;        // queries per GEMM tile (= TMEM lanes)
+
+// Candidates kept per query by the GEMM path before the exact re-ranking: k plus a margin of 3,
+// rounded up to a list length the select kernel is compiled for.
+__host__ __device__ inline int gemm_list_len(int k) {
+    int want = k + 3;
+    return want <= 4 ? 4 : want <= 8 ? 8 : want <= 16 ? 16 : 32;
+}
+
+// How the tiles of the distance GEMM are spread over the CTAs.  Query tiles (128 rows each) are taken in
+// groups of `mg`; inside a group, CTA (m_local, q) owns query tile m_local and the q-th of `parts` equal
+// ranges of cache rows, so CTAs with the same q stream the same cache rows at the same time (they meet in
+// L2) and each query row ends up with `parts` candidate lists.
+struct GemmPlan {
+    int32_t count;      // actual batch
+    int32_t m_tiles;    // ceil(count / 128)
+    int32_t mg;         // query tiles per group
+    int32_t groups;     // ceil(m_tiles / mg)
+    int32_t parts;      // cache-row ranges per query tile = candidate lists per query
+    int32_t range16;    // rows per range, in units of 16 (the last range may be shorter)
+    int32_t list_len;   // entries per candidate list
+    int32_t pad;
+};
+
+__host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entries, int num_ctas, int k) {
+    GemmPlan p;
+    p.count = count;
+    p.m_tiles = (count + kTileM - 1) / kTileM;
+    p.list_len = gemm_list_len(k);
+    p.pad = 0;
+    long long n16 = (n_entries + 15) / 16;
+    if (p.m_tiles <= 0 || n16 <= 0) {
+        p.mg = p.groups = p.parts = 1;
+        p.range16 = 0;
+        return p;
+    }
+    // pick the group size that needs the fewest MMA columns per CTA in total
+    int best_mg = 1;
+    long long best_cost = -1;
+    int mg_max = p.m_tiles < 16 ? p.m_tiles : 16;
+    if (mg_max > num_ctas) mg_max = num_ctas;
+    for (int mg = 1; mg <= mg_max; ++mg) {
+        int groups = (p.m_tiles + mg - 1) / mg;
+        int mg_eff = (p.m_tiles + groups - 1) / groups;
+        long long parts = num_ctas / mg_eff;
+        if (parts > n16) parts = n16;
+        long long r16 = (n16 + parts - 1) / parts;
+        long long cost = (long long)groups * r16;
+        if (best_cost < 0 || cost < best_cost || (cost == best_cost && mg_eff > best_mg)) {
+            best_cost = cost;
+            best_mg = mg_eff;
+        }
+    }
+    p.mg = best_mg;
+    p.groups = (p.m_tiles + p.mg - 1) / p.mg;
+    long long parts = num_ctas / p.mg;
+    if (parts > n16) parts = n16;
+    long long r16 = (n16 + parts - 1) / parts;
+    parts = (n16 + r16 - 1) / r16;   // drop ranges that would be empty
+    p.parts = (int32_t)parts;
+    p.range16 = (int32_t)r16;
+    return p;
+}
+
+struct LaunchCtx {
+    cudaStream_t stream;
+};
+
+}  // namespace fi
+
+// The cache object behind the opaque handle.
+struct fi_cache {
+    fi_cache_config_t cfg;
+    int64_t size;            // entries stored
+    int sm_count;
+    size_t elem_size;
+    // device storage owned by the cache
+    void *rows;              // [capacity x dim]
+    int32_t *labels;         // [capacity]
+    float *weights;          // [capacity]
+    float *norms;            // [capacity] squared norms of the stored values (fp32)
+    // look-up scratch
+    float *part_score;       // candidate lists
+    int32_t *part_idx;
+    size_t part_entries;     // capacity of the two arrays, in entries
+    void *q_compact;         // [max_batch x dim] gathered queries for the GEMM path (bf16 caches)
+    int32_t *slot_label;     // [max_batch] per-slot results of a cascade step
+    float *slot_conf;
+    uint8_t *slot_hit;
+    fi::GemmPlan *plan_dev;  // written by the GEMM kernel, read by the finalize kernel
+    int32_t *status_dev;     // device status word (bounded waits that ran out)
+    // staging for the host-buffer entry points (allocated on first use)
+    void *h2d_stage;
+    size_t h2d_stage_bytes;
+    int32_t *casc_buf;       // device arrays of a host-driven cascade
+    size_t casc_buf_batch;
+    // tensor maps over the cache rows (bf16 only): boxes of 64 and of 16 rows by 64 elements
+    CUtensorMap tmap_rows64;
+    CUtensorMap tmap_rows16;
+    bool tmaps_ready;
+};
+
+namespace fi {
+
+void set_error(const char *fmt, ...);
+void count_launch(int n = 1);
+fi_status_t check_launch(const char *what);
+
+// ---- launchers (each enqueues on `stream`, returns a status) ----
+fi_status_t launch_row_norms(const void *rows, int dtype, int64_t n, int dim, float *norms, cudaStream_t stream);
+
+fi_status_t launch_gather_rows(const void *src, int64_t ld_elems, const int32_t *row_idx, int32_t batch_max,
+                               const int32_t *count_dev, void *dst, int dim, size_t elem_size, cudaStream_t stream);
+
+// streaming look-up: writes candidate lists [batch][parts][k] (exact fp32 squared distances); returns parts
+fi_status_t launch_stream_lookup(const fi_cache *c, const void *queries, int64_t ld_elems, const int32_t *row_idx,
+                                 int32_t batch_max, const int32_t *count_dev, int *parts_out, cudaStream_t stream);
+
+// tensor-core distance GEMM with fused per-row select: writes candidate lists [batch][parts][list_len] of
+// scores ||c||^2 - 2 q.c and the plan it used to c->plan_dev
+fi_status_t launch_gemm_select(fi_cache *c, const void *queries_compact, int64_t ld_elems, int32_t batch_max,
+                               const int32_t *count_dev, cudaStream_t stream);
+
+// merge candidate lists, (optionally) recompute exact distances, vote, hit
+struct FinalizeArgs {
+    const void *queries;
+    int64_t ld_elems;
+    const int32_t *row_idx;
+    int32_t batch_max;
+    const int32_t *count_dev;
+    int parts;              // lists per query, or -1: read from plan_dev
+    int list_len;           // entries per list, or -1: read from plan_dev
+    int refine;             // 1: scores are approximate, recompute sum (q-c)^2 for the candidates
+    fi_lookup_out_t out;
+};
+fi_status_t launch_finalize(const fi_cache *c, const FinalizeArgs &a, cudaStream_t stream);
+
+fi_status_t launch_compact(const fi_cache *c, const fi_cascade_state_t &st, cudaStream_t stream);
+fi_status_t launch_cascade_init(const fi_cascade_state_t &st, int32_t num_stages, cudaStream_t stream);
+
+fi_status_t ensure_tensor_maps(fi_cache *c);
+size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k);
+
+}  // namespace fi

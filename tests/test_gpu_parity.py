@@ -1,0 +1,329 @@
+"""CUDA path vs fp64 oracle through the C ABI, element by element, on seeded inputs small enough for the
+oracle to finish in seconds but spanning several tiles, ragged tails and the degenerate cases."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fi_oracle as fo
+from paper_2002_02645_b200 import binding as fb
+from paper_2002_02645_b200 import datagen as dg
+from helpers import compare_lookup, f32, make_cache, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def run_lookup(cache, queries_np, **kw):
+    q = to_device(queries_np, cache.device)
+    out = cache.lookup_batch(q, **kw)
+    torch.cuda.synchronize()
+    cache.poll_status()
+    return (out.label.cpu().numpy(), out.conf.cpu().numpy(), out.hit.cpu().numpy(), out.topk_dist.cpu().numpy(),
+            out.topk_idx.cpu().numpy())
+
+
+def check_case(stage, *, k, num_classes, rule, path, percentile=50.0, metric=0, weights=None, twice=True):
+    storage = stage.dtype
+    ref0 = fo.lookup(stage.queries, stage.cache_vecs, stage.cache_labels, k=k, tau=0.0, rule=rule, metric=metric,
+                     weights=weights)
+    if rule == fo.RULE_CONF_GT:
+        finite = ref0.conf[np.isfinite(ref0.conf)]
+        tau = f32(np.percentile(finite, percentile)) if finite.size else 1.0
+    else:
+        tau = f32(np.percentile(ref0.nd[:, 0], percentile))
+    ref = fo.lookup(stage.queries, stage.cache_vecs, stage.cache_labels, k=k, tau=tau, rule=rule, metric=metric,
+                    weights=weights)
+    cache = make_cache(stage, k=k, num_classes=num_classes, rule=rule, metric=metric, tau=tau,
+                       max_batch=max(stage.queries.shape[0], 1), path=path, weights=weights)
+    got = run_lookup(cache, stage.queries)
+    stats = compare_lookup(*got, ref, storage=storage, tau=tau, rule=rule, metric=metric,
+                           cache_labels=stage.cache_labels, weights=weights)
+    if twice:   # a race would show as run-to-run differences
+        again = run_lookup(cache, stage.queries)
+        for a, b in zip(got, again):
+            np.testing.assert_array_equal(a, b)
+    print(stats)
+    assert stats.exempt_gap <= max(2, stage.queries.shape[0] // 5)
+    assert 0 < ref.hit.sum() < ref.hit.shape[0] or stage.queries.shape[0] < 4
+    cache.close()
+    return stats
+
+
+# ------------------------------------------------------------------ config 1: fp32, k = 1, exact copies, DIST_LE
+
+def test_config1_full():
+    w = dg.config1(seed=0)
+    st = w.stages[0]
+    x64 = st.cache_vecs.astype(np.float64)
+    # 20th percentile of squared distances between distinct cache entries of equal label
+    d = []
+    for c in range(10):
+        xc = x64[st.cache_labels == c]
+        D = ((xc[:, None, :] - xc[None, :, :]) ** 2).sum(-1)
+        d.append(D[np.triu_indices(xc.shape[0], 1)])
+    tau = f32(np.percentile(np.concatenate(d), 20.0))
+    ref = fo.lookup(st.queries, st.cache_vecs, st.cache_labels, k=1, tau=tau, rule=fo.RULE_DIST_LE)
+    cache = make_cache(st, k=1, num_classes=10, rule=fb.FI_HIT_DIST_LE, tau=tau, max_batch=282)
+    got = run_lookup(cache, st.queries)
+    stats = compare_lookup(*got, ref, storage="f32", tau=tau, rule=1, cache_labels=st.cache_labels)
+    print(stats)
+    copies = w.meta["copy_of"] >= 0
+    assert (got[3][copies, 0] == 0).all() and np.isinf(got[1][copies]).all() and (got[2][copies] == 1).all()
+    np.testing.assert_array_equal(got[4][copies, 0], w.meta["copy_of"][copies])
+    assert stats.exempt_gap == 0 and ref.hit.sum() >= 26
+    cache.close()
+
+
+# ------------------------------------------------------------------ streaming path, bf16 and fp32, ragged shapes
+
+@pytest.mark.parametrize("n,d,b,k,dtype", [
+    (777, 520, 1, 1, "bf16"), (777, 520, 3, 5, "bf16"), (1501, 64, 4, 10, "bf16"), (333, 2048, 2, 1, "bf16"),
+    (9, 8, 4, 5, "bf16"), (1000, 36, 37, 3, "f32"), (257, 4, 5, 32, "f32"), (4100, 16384, 4, 1, "bf16")])
+def test_stream_path(n, d, b, k, dtype):
+    w = dg.single_layer(name="t", n_cache=n, n_query=b, dim=d, num_classes=7, dtype=dtype, sigma=0.5, k=k, seed=3)
+    check_case(w.stages[0], k=k, num_classes=7, rule=fo.RULE_CONF_GT, path=fb.FI_PATH_STREAM)
+
+
+def test_stream_path_large_dim_reads_queries_in_place():
+    # 4 query rows of 65536 bf16 values do not fit in shared memory
+    w = dg.single_layer(name="t", n_cache=300, n_query=4, dim=65536, num_classes=5, dtype="bf16", sigma=0.5, k=2, seed=4)
+    check_case(w.stages[0], k=2, num_classes=5, rule=fo.RULE_CONF_GT, path=fb.FI_PATH_STREAM)
+
+
+# ------------------------------------------------------------------ tensor-core path: several tiles, ragged M, N, K
+
+@pytest.mark.parametrize("n,d,b,k", [
+    (5003, 200, 300, 5),       # 3 query tiles (last ragged), ragged N, K = 3 blocks + 8
+    (40000, 64, 129, 10),      # one k-block, many row ranges, 2 query tiles
+    (600, 1024, 5, 1),         # tiny batch, fewer 16-row blocks than CTAs
+    (16, 8, 17, 5),            # a single 16-row block
+    (3000, 4096, 64, 13),      # list length 16, deep K
+    (2500, 136, 2200, 29),     # 18 query tiles (two groups), list length 32
+])
+def test_gemm_path(n, d, b, k):
+    w = dg.single_layer(name="t", n_cache=n, n_query=b, dim=d, num_classes=9, dtype="bf16", sigma=0.6, k=k, seed=5)
+    check_case(w.stages[0], k=k, num_classes=9, rule=fo.RULE_CONF_GT, path=fb.FI_PATH_GEMM)
+
+
+def test_gemm_and_stream_paths_agree_and_copies_hit():
+    w = dg.single_layer(name="t", n_cache=3000, n_query=40, dim=512, num_classes=6, dtype="bf16", sigma=0.5, k=5,
+                        seed=6, n_copies=8)
+    st = w.stages[0]
+    ref = fo.lookup(st.queries, st.cache_vecs, st.cache_labels, k=5, tau=1e30)
+    outs = []
+    for path in (fb.FI_PATH_STREAM, fb.FI_PATH_GEMM):
+        cache = make_cache(st, k=5, num_classes=6, tau=1e30, max_batch=48, path=path)
+        got = run_lookup(cache, st.queries)
+        compare_lookup(*got, ref, storage="bf16", tau=1e30, rule=0, cache_labels=st.cache_labels)
+        outs.append(got)
+        cache.close()
+    copies = w.meta["copy_of"] >= 0
+    for got in outs:   # observation O1: an identical activation freezes, whatever the threshold
+        assert (got[3][copies, 0] == 0).all() and np.isinf(got[1][copies]).all() and (got[2][copies] == 1).all()
+        assert (got[2][~copies] == 0).all()
+    np.testing.assert_array_equal(outs[0][0], outs[1][0])
+    np.testing.assert_array_equal(outs[0][4], outs[1][4])
+
+
+def test_kmeans_entries_weights_and_l2_metric():
+    # Sec. 4: entries <centre, majority label, fraction>; k = 1 gives confidence f / distance
+    w = dg.single_layer(name="t", n_cache=200, n_query=64, dim=1024, num_classes=10, dtype="bf16", sigma=0.5, k=1, seed=7)
+    frac = np.random.default_rng(0).uniform(0.4, 1.0, 200).astype(np.float32)
+    for path in (fb.FI_PATH_STREAM, fb.FI_PATH_GEMM):
+        for metric in (0, 1):
+            check_case(w.stages[0], k=1, num_classes=10, rule=fo.RULE_CONF_GT, path=path, metric=metric, weights=frac)
+    check_case(w.stages[0], k=4, num_classes=10, rule=fo.RULE_DIST_LE, path=fb.FI_PATH_GEMM, metric=1, weights=frac)
+
+
+# ------------------------------------------------------------------ degenerate cases
+
+def test_empty_cache_k_above_size_and_zero_batch():
+    w = dg.single_layer(name="t", n_cache=3, n_query=6, dim=64, num_classes=4, dtype="bf16", sigma=0.5, k=5, seed=8)
+    st = w.stages[0]
+    ref = fo.lookup(st.queries, st.cache_vecs, st.cache_labels, k=5, tau=0.0)
+    for path in (fb.FI_PATH_STREAM, fb.FI_PATH_GEMM):
+        cache = make_cache(st, k=5, num_classes=4, tau=0.0, max_batch=8, path=path, capacity=10)
+        got = run_lookup(cache, st.queries)
+        compare_lookup(*got, ref, storage="bf16", tau=0.0, rule=0, cache_labels=st.cache_labels)
+        assert (got[4][:, 3:] == -1).all()
+        cache.close()
+    empty = fb.FreezeCache(dim=64, capacity=10, num_classes=4, k=5, dtype=fb.FI_BF16, max_batch=8)
+    got = run_lookup(empty, st.queries)
+    assert (got[0] == -1).all() and (got[1] == 0).all() and (got[2] == 0).all() and (got[4] == -1).all()
+    # batch 0: nothing is launched, nothing is written
+    q = to_device(st.queries, empty.device)
+    out = fb.LookupOut(1, 5, empty.device)
+    out.label.fill_(77)
+    empty.lookup_batch(q[:0], batch_max=0, out=out)
+    torch.cuda.synchronize()
+    assert int(out.label[0]) == 77
+    empty.close()
+
+
+def test_gather_list_and_device_resident_count():
+    w = dg.single_layer(name="t", n_cache=2000, n_query=300, dim=256, num_classes=5, dtype="bf16", sigma=0.5, k=5, seed=9)
+    st = w.stages[0]
+    rows = np.sort(np.random.default_rng(1).choice(300, 150, replace=False)).astype(np.int32)
+    for path, count in ((fb.FI_PATH_GEMM, 131), (fb.FI_PATH_STREAM, 3), (fb.FI_PATH_GEMM, 0)):
+        cache = make_cache(st, k=5, num_classes=5, tau=0.05, max_batch=150, path=path)
+        ref = fo.lookup(st.queries, st.cache_vecs, st.cache_labels, k=5, tau=f32(0.05), row_idx=rows[:count])
+        out = fb.LookupOut(150, 5, cache.device)
+        out.label.fill_(-7)
+        cnt = torch.tensor([count], dtype=torch.int32, device=cache.device)
+        cache.lookup_batch(to_device(st.queries, cache.device), row_idx=torch.from_numpy(rows).to(cache.device),
+                           batch_max=150, batch_count=cnt, out=out)
+        torch.cuda.synchronize()
+        cache.poll_status()
+        lab = out.label.cpu().numpy()
+        assert (lab[count:] == -7).all()      # slots past the actual batch stay untouched
+        if count:
+            compare_lookup(lab[:count], out.conf.cpu().numpy()[:count], out.hit.cpu().numpy()[:count],
+                           out.topk_dist.cpu().numpy()[:count], out.topk_idx.cpu().numpy()[:count], ref, storage="bf16",
+                           tau=f32(0.05), rule=0, cache_labels=st.cache_labels)
+        cache.close()
+
+
+def test_strided_queries_and_incremental_insert():
+    w = dg.single_layer(name="t", n_cache=900, n_query=20, dim=128, num_classes=5, dtype="bf16", sigma=0.5, k=3, seed=10)
+    st = w.stages[0]
+    ref = fo.lookup(st.queries, st.cache_vecs, st.cache_labels, k=3, tau=0.0)
+    for path in (fb.FI_PATH_STREAM, fb.FI_PATH_GEMM):
+        cache = fb.FreezeCache(dim=128, capacity=1000, num_classes=5, k=3, dtype=fb.FI_BF16, max_batch=32, path=path)
+        xs, ls = to_device(st.cache_vecs), torch.from_numpy(st.cache_labels).cuda()
+        for lo, hi in ((0, 1), (1, 450), (450, 900)):     # Sec. 5: entries can be appended later
+            cache.insert(xs[lo:hi].contiguous(), ls[lo:hi].contiguous())
+        assert cache.size() == 900
+        wide = torch.zeros(20, 256, dtype=torch.bfloat16, device="cuda")
+        wide[:, :128] = to_device(st.queries)
+        out = cache.lookup_batch(wide[:, :128])              # leading dimension 256
+        torch.cuda.synchronize()
+        compare_lookup(out.label.cpu().numpy(), out.conf.cpu().numpy(), out.hit.cpu().numpy(),
+                       out.topk_dist.cpu().numpy(), out.topk_idx.cpu().numpy(), ref, storage="bf16", tau=0.0, rule=0,
+                       cache_labels=st.cache_labels)
+        cache.close()
+
+
+def test_error_statuses():
+    with pytest.raises(fb.FiError) as e:
+        fb.FreezeCache(dim=12, capacity=10, num_classes=4, k=5, dtype=fb.FI_BF16)      # dim not a multiple of 8
+    assert e.value.status == 1
+    with pytest.raises(fb.FiError) as e:
+        fb.FreezeCache(dim=16, capacity=10, num_classes=4, k=33, dtype=fb.FI_BF16)     # k above 32
+    assert e.value.status == 1
+    with pytest.raises(fb.FiError) as e:
+        fb.FreezeCache(dim=16, capacity=10, num_classes=4, k=3, dtype=fb.FI_F32, path=fb.FI_PATH_GEMM)
+    assert e.value.status == 5
+    c = fb.FreezeCache(dim=16, capacity=4, num_classes=4, k=1, dtype=fb.FI_BF16, max_batch=4)
+    x = torch.zeros(5, 16, dtype=torch.bfloat16, device="cuda")
+    lab = torch.zeros(5, dtype=torch.int32, device="cuda")
+    with pytest.raises(fb.FiError) as e:
+        c.insert(x, lab)                                                                  # beyond capacity
+    assert e.value.status == 2 and c.size() == 0
+    with pytest.raises(fb.FiError) as e:
+        c.lookup_batch(x)                                                                 # batch above max_batch
+    assert e.value.status == 1
+    c.close()
+
+
+# ------------------------------------------------------------------ cascades
+
+def oracle_taus(w):
+    taus = []
+    for s, p in zip(w.stages, w.meta["percentiles"]):
+        c = fo.lookup(s.calib, s.cache_vecs, s.cache_labels, k=w.k, tau=0.0).conf
+        taus.append(f32(np.percentile(c, p)))
+    return taus
+
+
+def run_cascade_device(w, taus, path):
+    b0 = w.stages[0].queries.shape[0]
+    caches = [make_cache(s, k=w.k, num_classes=w.num_classes, tau=t, max_batch=b0, path=path)
+              for s, t in zip(w.stages, taus)]
+    acts = [to_device(s.queries) for s in w.stages]
+    state = fb.CascadeState(b0, "cuda:0")
+    fb.cascade_init(state, len(caches))
+    survivors = []
+    for l, (c, a) in enumerate(zip(caches, acts)):
+        fb.cascade_step(c, a, state, l)
+        ids, cnt = state.survivors(l)
+        torch.cuda.synchronize()
+        survivors.append(ids[: int(cnt.item())].cpu().numpy().copy())
+    for c in caches:
+        c.poll_status()
+    res = (state.final_label.cpu().numpy()[:b0], state.exit_stage.cpu().numpy()[:b0],
+           state.final_conf.cpu().numpy()[:b0], survivors)
+    return caches, res
+
+
+def check_cascade(w, path):
+    taus = oracle_taus(w)
+    ref = fo.cascade([s.queries for s in w.stages], [s.cache_vecs for s in w.stages],
+                     [s.cache_labels for s in w.stages], taus, k=w.k)
+    caches, (label, stage, conf, survivors) = run_cascade_device(w, taus, path)
+    # requests whose neighbour set / vote / threshold test is not decidable at some stage they reached
+    undecidable = np.zeros(label.shape[0], bool)
+    for l, r in enumerate(ref.stage_results):
+        ids = ref.active[l]
+        kth = r.nd[:, -1]
+        gap = (r.next_d - kth) / kth
+        near = np.abs(r.conf - taus[l]) / taus[l] < 1e-5
+        undecidable[ids[(gap < 1e-4) | near]] = True
+    print(f"{w.name}: arrivals {[a.shape[0] for a in ref.active]}, undecidable {int(undecidable.sum())}")
+    if not undecidable.any():
+        for l in range(len(w.stages)):
+            np.testing.assert_array_equal(survivors[l], ref.active[l + 1])       # miss_idx and miss_count, bit-exact
+        np.testing.assert_array_equal(label, ref.final_label)
+        np.testing.assert_array_equal(stage, ref.exit_stage)
+    else:
+        ok = ~undecidable
+        np.testing.assert_array_equal(label[ok], ref.final_label[ok])
+        np.testing.assert_array_equal(stage[ok], ref.exit_stage[ok])
+    frozen = ref.exit_stage < len(w.stages)
+    ok = frozen & ~undecidable
+    np.testing.assert_allclose(conf[ok], ref.final_conf[ok], rtol=1e-2)
+    for l in range(len(w.stages)):
+        assert (np.diff(survivors[l]) > 0).all()
+    assert ref.active[-1].shape[0] > 0 and (ref.exit_stage == 0).sum() > 0
+    # the host-buffer entry point gives the same answers
+    from helpers import to_host_tensor
+    b0 = label.shape[0]
+    hl = torch.empty(b0, dtype=torch.int32).pin_memory()
+    hs = torch.empty(b0, dtype=torch.int32).pin_memory()
+    hc = torch.empty(b0, dtype=torch.float32).pin_memory()
+    arr = torch.zeros(len(caches) + 1, dtype=torch.int32).pin_memory()
+    fb.cascade_run_host(caches, [to_host_tensor(s.queries, pin=True) for s in w.stages], hl, hs, hc, arr)
+    np.testing.assert_array_equal(hl.numpy(), label)
+    np.testing.assert_array_equal(hs.numpy(), stage)
+    np.testing.assert_array_equal(hc.numpy(), conf)
+    np.testing.assert_array_equal(arr.numpy(), [b0] + [s.shape[0] for s in survivors])
+    for c in caches:
+        c.close()
+
+
+@pytest.mark.parametrize("path", [fb.FI_PATH_GEMM, fb.FI_PATH_STREAM])
+def test_cascade_resnet18_shape_shrunk(path):
+    check_cascade(dg.config2(seed=0, shrink=16), path)
+
+
+def test_cascade_imagenet_shape_shrunk():
+    check_cascade(dg.config4(seed=0, shrink=8), fb.FI_PATH_GEMM)
+
+
+def test_cascade_threshold_limits():
+    w = dg.config2(seed=0, shrink=32)
+    _, (label, stage, _, surv) = run_cascade_device(w, [float("inf")] * 4, fb.FI_PATH_GEMM)
+    assert (stage == 4).all() and (label == -1).all() and all(s.shape[0] == 32 for s in surv)
+    _, (label, stage, _, surv) = run_cascade_device(w, [0.0] * 4, fb.FI_PATH_GEMM)
+    assert (stage == 0).all() and all(s.shape[0] == 0 for s in surv)
+
+
+def test_host_lookup_matches_device_lookup():
+    from helpers import to_host_tensor
+    w = dg.single_layer(name="t", n_cache=1200, n_query=70, dim=256, num_classes=5, dtype="bf16", sigma=0.5, k=5, seed=12)
+    st = w.stages[0]
+    cache = make_cache(st, k=5, num_classes=5, tau=0.02, max_batch=70)
+    dev = run_lookup(cache, st.queries)
+    out = fb.LookupOut(70, 5, "cpu")
+    cache.lookup_batch_host(to_host_tensor(st.queries, pin=True), out)
+    for a, b in zip(dev, (out.label, out.conf, out.hit, out.topk_dist, out.topk_idx)):
+        np.testing.assert_array_equal(a, b.numpy())
+    cache.close()
