@@ -1,0 +1,438 @@
+#!/usr/bin/env python
+"""Throughput of the per-layer cache look-up on B200: one JSON line per run.
+
+A step is one pass of the whole hot path over one batch of synthetic requests.  The default workload is the
+four-stage ResNet-18/CIFAR-10-shaped cascade (bf16 caches of 10,000 entries with 65536 / 32768 / 16384 / 8192
+values per entry, batch 1,024, k = 5, misses compacted between stages); `--workload` also offers the large-cache
+layer (200,000 x 8192, batch 8,192, k = 10) and the latency layer (50,000 x 16384, batch 1 / 4 / 16, k = 1).
+
+`value` is queries/s with every input already resident in HBM; `e2e` is the same metric through the host-buffer
+entry point of the C ABI (pinned host activations copied in, results copied out, every step).  With --gpus N
+every rank holds its own caches and its own batch (the look-ups of different requests are independent, so
+ranks never exchange data): weak scaling.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg5] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "cache-lookup queries/sec per layer (1 B200) and % of bf16 TC peak / HBM BW"
+UNIT = "queries/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"]))}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                smax.append(float(r[1]))
+                for name, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                continue
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        busy = [v for v in sm if v > 0.5 * max(sm)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    return rank, local, world
+
+
+# ---------------------------------------------------------------------------------------------- workloads
+
+def build_workload(name: str, seed: int, query_seed=None):
+    from paper_2002_02645_b200 import datagen as dg
+    if name == "cfg2":
+        return dg.config2(seed=seed, query_seed=query_seed)
+    if name == "cfg3":
+        return dg.config3(seed=seed, query_seed=query_seed)
+    if name == "cfg5":
+        return dg.config5(seed=seed, batch=16, query_seed=query_seed)
+    if name == "cfg2-small":       # same recipe, 1/16 of the sizes: a quick functional run
+        return dg.config2(seed=seed, shrink=16, query_seed=query_seed)
+    if name == "cfg2-s0":          # first stage of cfg2 alone (10,000 x 65536, batch 1,024): the dominant GEMM
+        w = dg.config2(seed=seed, query_seed=query_seed, stages=1)
+        w.name = "cfg2_stage0_only"
+        return w
+    raise SystemExit(f"unknown workload {name}")
+
+
+def to_dev(a, dev):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    return t.view(torch.int16).to(dev).view(torch.bfloat16) if a.dtype == np.uint16 else t.to(dev)
+
+
+def to_pinned(a):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if a.dtype == np.uint16:
+        t = t.view(torch.int16).view(torch.bfloat16)
+    return t.pin_memory()
+
+
+def calibrate(cache, calib_dev, percentile):
+    """THRESHOLDS[layer] for the synthetic data: the given percentile of the confidences the library itself
+    returns for a separate calibration batch (offline phase, Sec. 3.1 (ii), with a percentile in place of the
+    validation-error rule because synthetic requests have no model prediction to disagree with)."""
+    import torch
+    cache.set_threshold(0.0)
+    out = cache.lookup_batch(calib_dev, with_topk=False)
+    torch.cuda.synchronize()
+    conf = out.conf.cpu().numpy().astype(np.float64)
+    conf = conf[np.isfinite(conf)]
+    tau = float(np.float32(np.percentile(conf, percentile)))
+    cache.set_threshold(tau)
+    return tau
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2002_02645_b200 import binding as fb
+    from paper_2002_02645_b200 import build as fbuild
+
+    rank, local, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        fbuild.build_library()
+    if world > 1:
+        dist.barrier()
+    fb.load_library()
+
+    t_gen = time.time()
+    # every rank serves its own requests: same caches, batch drawn from the rank's own seed
+    w = build_workload(args.workload, seed=0, query_seed=None if (rank == 0 or args.same_batch) else 1000 + rank)
+    t_gen = time.time() - t_gen
+
+    n_stage = len(w.stages)
+    b0 = w.stages[0].queries.shape[0]
+    cascade = n_stage > 1
+    rule = fb.FI_HIT_CONF_GT if w.meta.get("rule", "conf_gt") == "conf_gt" else fb.FI_HIT_DIST_LE
+    caches, acts, taus = [], [], []
+    for s_i, st in enumerate(w.stages):
+        c = fb.FreezeCache(dim=st.dim, capacity=st.cache_vecs.shape[0], num_classes=w.num_classes, k=w.k,
+                           dtype=fb.FI_BF16 if st.dtype == "bf16" else fb.FI_F32, rule=rule, device=local,
+                           max_batch=max(b0, 0 if st.calib is None else st.calib.shape[0]))
+        # insert in slices so the staging copy on the device stays small
+        n = st.cache_vecs.shape[0]
+        step_rows = max(1, (512 << 20) // (st.dim * 2))
+        for lo in range(0, n, step_rows):
+            hi = min(n, lo + step_rows)
+            c.insert(to_dev(st.cache_vecs[lo:hi], dev), torch.from_numpy(st.cache_labels[lo:hi]).to(dev))
+        torch.cuda.synchronize()
+        if rule == fb.FI_HIT_CONF_GT and st.calib is not None:
+            taus.append(calibrate(c, to_dev(st.calib, dev), w.meta["percentiles"][s_i]))
+        else:
+            # fixed threshold: 20th percentile of nearest-neighbour squared distances of the batch itself
+            c.set_threshold(float("inf"))
+            out = c.lookup_batch(to_dev(st.queries, dev))
+            torch.cuda.synchronize()
+            tau = float(np.float32(np.percentile(out.topk_dist[:, 0].cpu().numpy(), 20.0)))
+            c.set_threshold(tau)
+            taus.append(tau)
+        caches.append(c)
+        acts.append(to_dev(st.queries, dev))
+
+    state = fb.CascadeState(b0, dev)
+    out_single = fb.LookupOut(b0, w.k, dev, with_topk=False)
+
+    def step():
+        if cascade:
+            fb.cascade_init(state, n_stage)
+            for l in range(n_stage):
+                fb.cascade_step(caches[l], acts[l], state, l)
+        else:
+            caches[0].lookup_batch(acts[0], out=out_single)
+
+    def fence():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    fence()
+    for c in caches:
+        c.poll_status()
+
+    # per-stage arrivals (what the cascade actually does on this data): one extra pass, read after every stage
+    arrivals = [b0]
+    if cascade:
+        fb.cascade_init(state, n_stage)
+        for l in range(n_stage):
+            fb.cascade_step(caches[l], acts[l], state, l)
+            arrivals.append(int(state.survivors(l)[1].item()))
+        fence()
+
+    for c in caches:
+        c.set_profiling(True)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    launches0 = fb.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    fence()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    fence()
+    launches = fb.launch_count() - launches0
+    ms_total = ev0.elapsed_time(ev1)
+    clocks = sampler.stop()
+    prof = [c.read_profile() for c in caches]
+    for c in caches:
+        c.set_profiling(False)
+        c.poll_status()
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = world * b0 * args.steps / (ms_total * 1e-3)
+
+    # ---- end to end through the host-buffer entry point
+    host_acts = [to_pinned(st.queries) for st in w.stages]
+    h_label = torch.empty(b0, dtype=torch.int32).pin_memory()
+    h_stage = torch.empty(b0, dtype=torch.int32).pin_memory()
+    h_conf = torch.empty(b0, dtype=torch.float32).pin_memory()
+    h_out = fb.LookupOut(b0, w.k, "cpu", with_topk=False)
+    for name in ("label", "conf", "hit"):
+        setattr(h_out, name, getattr(h_out, name).pin_memory())
+
+    def e2e_step():
+        if cascade:
+            fb.cascade_run_host(caches, host_acts, h_label, h_stage, h_conf)
+        else:
+            caches[0].lookup_batch_host(host_acts[0], h_out)
+
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        e2e_step()
+    fence()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    fence()
+    e2e_s = time.perf_counter() - t0
+    t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_s = float(t.item())
+    h2d = sum(int(a.numel() * a.element_size()) for a in host_acts)
+    d2h = b0 * 12 if cascade else b0 * 9
+    e2e = {"value": world * b0 * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": 1e3 * e2e_s / e2e_steps}
+
+    # ---- roofline of the dominant kernel: the distance kernel of the first (largest) stage
+    peaks, peak_src = load_peaks()
+    st0 = w.stages[0]
+    n0, d0 = st0.cache_vecs.shape
+    ms0, n_launch0 = prof[0]
+    roofline = None
+    if n_launch0 > 0 and ms0 > 0:
+        avg_s = ms0 / n_launch0 * 1e-3
+        if b0 > 4:
+            flops = 2.0 * b0 * n0 * d0
+            achieved = flops / avg_s / 1e12
+            roofline = {"bound": "tensor", "kernel": "gemm_select_kernel (stage 0)", "achieved": achieved,
+                        "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                        "peak_source": f"bf16 burst, {peak_src}", "traffic": None,
+                        "avg_launch_ms": avg_s * 1e3, "launches": n_launch0}
+        else:
+            nbytes = n0 * d0 * 2.0 + b0 * d0 * 2.0
+            achieved = nbytes / avg_s / 1e9
+            roofline = {"bound": "hbm", "kernel": "stream_lookup_kernel", "achieved": achieved,
+                        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                        "peak_source": f"copy bandwidth, {peak_src}", "traffic": None,
+                        "avg_launch_ms": avg_s * 1e3, "launches": n_launch0}
+    stage_info = []
+    for l, (ms_l, n_l) in enumerate(prof):
+        if n_l:
+            nl, dl = w.stages[l].cache_vecs.shape
+            bl = arrivals[l] if cascade else b0
+            stage_info.append({"stage": l, "arrivals": bl, "distance_kernel_ms": ms_l / n_l,
+                               "tflops": 2.0 * bl * nl * dl / (ms_l / n_l * 1e-3) / 1e12})
+
+    # ---- the oracle on the host cores, bounded sample (rank 0, single GPU runs only)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = time_oracle(w, taus, args.cpu_sample)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if st0.dtype == "bf16" else "f32",
+                "data": "synthetic",
+                "config": {"workload": w.name, "stages": n_stage, "batch": b0, "k": w.k,
+                           "cache_entries": int(n0), "dims": [s.dim for s in w.stages],
+                           "thresholds": taus, "arrivals": arrivals,
+                           "l2": "inputs larger than L2 (caches %.2f GB)" % (sum(s.cache_vecs.nbytes for s in w.stages) / 1e9),
+                           "parallelism": f"replicas x{world}", "datagen_s": round(t_gen, 1)},
+                "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
+                "stages": stage_info, "cpu_baseline": cpu_baseline}
+        print(json.dumps(line))
+    for c in caches:
+        c.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------------- CPU oracle leg
+
+def oracle_sample_step(w, taus, sample):
+    from oracle import fi_oracle as fo
+    rule = fo.RULE_CONF_GT if w.meta.get("rule", "conf_gt") == "conf_gt" else fo.RULE_DIST_LE
+    qs = [s.queries[:sample] for s in w.stages]
+    if len(w.stages) > 1:
+        fo.cascade(qs, [s.cache_vecs for s in w.stages], [s.cache_labels for s in w.stages], taus, k=w.k, rule=rule)
+    else:
+        s = w.stages[0]
+        fo.lookup(qs[0], s.cache_vecs, s.cache_labels, k=w.k, tau=taus[0], rule=rule)
+
+
+def default_cpu_sample(w, reference_arm=False):
+    """Requests whose oracle look-ups cost about 3e11 (baseline leg) or 5e10 (per reference step) multiply-adds."""
+    per_query = sum(s.cache_vecs.shape[0] * s.dim for s in w.stages)
+    budget = 5e10 if reference_arm else 3e11
+    return int(max(1, min(w.stages[0].queries.shape[0], budget // per_query)))
+
+
+def time_oracle(w, taus, sample):
+    cores = len(os.sched_getaffinity(0))
+    sample = min(sample or default_cpu_sample(w), w.stages[0].queries.shape[0])
+    t0 = time.perf_counter()
+    oracle_sample_step(w, taus, sample)
+    dt = time.perf_counter() - t0
+    return {"value": sample / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {sample} requests of the batch through all {len(w.stages)} stage(s) against the full "
+                      f"caches, fp64, OpenMP over queries; {dt:.1f} s"}
+
+
+def run_reference(args):
+    """The oracle as it stands, on the host cores, on a bounded sample of the same workload per step."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    w = build_workload(args.workload, seed=0)
+    from oracle import fi_oracle as fo
+    taus = []
+    for s, p in zip(w.stages, w.meta.get("percentiles", [50.0] * len(w.stages))):
+        if w.meta.get("rule", "conf_gt") == "conf_gt":
+            conf = fo.lookup(s.calib[:32], s.cache_vecs, s.cache_labels, k=w.k, tau=0.0).conf
+            taus.append(float(np.float32(np.percentile(conf, p))))
+        else:
+            taus.append(float("inf"))
+    sample = args.cpu_sample or default_cpu_sample(w, reference_arm=True)
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_step(w, taus, sample)
+    steps = max(1, min(args.steps, 3))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_sample_step(w, taus, sample)
+    dt = time.perf_counter() - t0
+    cores = len(os.sched_getaffinity(0))
+    value = sample * steps / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * dt / steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "stages": len(w.stages), "batch": sample, "k": w.k},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"first {sample} requests per step through all stages against the full caches"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg5", "cfg2-small", "cfg2-s0"])
+    ap.add_argument("--cpu-sample", type=int, default=0,
+                    help="requests per oracle timing (0: sized for 10-30 s of CPU work)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--same-batch", action="store_true", help="every rank serves the same batch")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -175,6 +175,16 @@ fi_status_t fi_cascade_run_host(fi_cache_t *const *stage_caches, int32_t num_sta
  * since the last poll (the word is cleared), FI_OK otherwise. */
 fi_status_t fi_cache_poll_status(fi_cache_t *cache);
 
+/*
+ * Device timing of the distance kernel (the tensor-core GEMM or the streaming kernel) of later look-ups on
+ * this cache: with profiling on, each look-up records a CUDA event before and after that kernel on the
+ * caller's stream (up to 256 look-ups are kept; older ones are overwritten).  fi_cache_read_profile
+ * synchronises on the recorded events, returns the summed kernel time in milliseconds and the number of
+ * launches it covers, and clears the record.  Events are created on first use and freed by destroy.
+ */
+fi_status_t fi_cache_set_profiling(fi_cache_t *cache, int32_t enable);
+fi_status_t fi_cache_read_profile(fi_cache_t *cache, float *total_ms, int32_t *launches);
+
 /* Number of kernels this library has launched in the calling process (all caches). */
 int64_t fi_launch_count(void);
 

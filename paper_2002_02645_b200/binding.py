@@ -22,7 +22,8 @@ FI_PATH_AUTO, FI_PATH_STREAM, FI_PATH_GEMM = 0, 1, 2
 
 EXPORTS = ["fi_cache_create", "fi_cache_destroy", "fi_cache_insert", "fi_cache_set_threshold", "fi_cache_set_path",
            "fi_cache_size", "fi_cache_lookup_batch", "fi_cascade_init", "fi_cascade_step", "fi_cache_lookup_batch_host",
-           "fi_cascade_run_host", "fi_cache_poll_status", "fi_launch_count", "fi_last_error", "fi_status_string"]
+           "fi_cascade_run_host", "fi_cache_poll_status", "fi_cache_set_profiling",
+           "fi_cache_read_profile", "fi_launch_count", "fi_last_error", "fi_status_string"]
 
 
 class fi_cache_config_t(ctypes.Structure):
@@ -75,6 +76,8 @@ def load_library(path: Optional[str] = None):
     lib.fi_cache_lookup_batch_host.argtypes = [vp, vp, i32, ctypes.POINTER(fi_lookup_out_t), vp]
     lib.fi_cascade_run_host.argtypes = [ctypes.POINTER(vp), i32, ctypes.POINTER(vp), i32, vp, vp, vp, vp, vp]
     lib.fi_cache_poll_status.argtypes = [vp]
+    lib.fi_cache_set_profiling.argtypes = [vp, i32]
+    lib.fi_cache_read_profile.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.fi_launch_count.argtypes = []
     lib.fi_launch_count.restype = i64
     lib.fi_last_error.argtypes = []
@@ -193,6 +196,16 @@ class FreezeCache:
 
     def poll_status(self) -> None:
         _check(self._lib.fi_cache_poll_status(self._h))
+
+    # -- fi_cache_set_profiling / fi_cache_read_profile
+    def set_profiling(self, enable: bool) -> None:
+        _check(self._lib.fi_cache_set_profiling(self._h, 1 if enable else 0))
+
+    def read_profile(self):
+        """(summed distance-kernel milliseconds, launches covered) since the last read."""
+        ms, n = ctypes.c_float(0.0), ctypes.c_int32(0)
+        _check(self._lib.fi_cache_read_profile(self._h, ctypes.byref(ms), ctypes.byref(n)))
+        return float(ms.value), int(n.value)
 
     # -- fi_cache_lookup_batch
     def lookup_batch(self, queries: torch.Tensor, *, row_idx: Optional[torch.Tensor] = None,

@@ -61,6 +61,18 @@ void free_all(fi_cache *c) {
     cudaFree(c->status_dev);
     cudaFree(c->h2d_stage);
     cudaFree(c->casc_buf);
+    if (c->prof_ev) {
+        for (int i = 0; i < 2 * kProfSlots; ++i) cudaEventDestroy(c->prof_ev[i]);
+        delete[] c->prof_ev;
+        c->prof_ev = nullptr;
+    }
+}
+
+// events around the distance kernel of one look-up
+void prof_mark(fi_cache *c, int which, cudaStream_t stream) {
+    if (!c->prof_on || !c->prof_ev) return;
+    cudaEventRecord(c->prof_ev[2 * (c->prof_n % kProfSlots) + which], stream);
+    if (which == 1) ++c->prof_n;
 }
 
 int resolve_path(const fi_cache *c, int batch_max) {
@@ -101,8 +113,10 @@ fi_status_t lookup_impl(fi_cache *c, const void *queries, int64_t ld, const int3
     fi_status_t st;
     if (path == FI_PATH_STREAM) {
         int parts = 1;
+        prof_mark(c, 0, stream);
         st = launch_stream_lookup(c, queries, ld, row_idx, batch_max, count_dev, &parts, stream);
         if (st != FI_OK) return st;
+        prof_mark(c, 1, stream);
         fa.parts = parts;
         fa.list_len = c->cfg.k;
         fa.refine = 0;
@@ -111,7 +125,7 @@ fi_status_t lookup_impl(fi_cache *c, const void *queries, int64_t ld, const int3
             set_error("the tensor-core path needs a bf16 cache");
             return FI_ERR_UNSUPPORTED;
         }
-        st = ensure_part_scratch(c, gemm_part_entries(batch_max, c->size, c->sm_count, c->cfg.k));
+        st = ensure_part_scratch(c, gemm_part_entries(batch_max, c->size, c->sm_count, c->cfg.k, c->cfg.dim));
         if (st != FI_OK) return st;
         const void *qsrc = queries;
         int64_t qld = ld;
@@ -124,8 +138,10 @@ fi_status_t lookup_impl(fi_cache *c, const void *queries, int64_t ld, const int3
             fa.ld_elems = qld;
             fa.row_idx = nullptr;
         }
+        prof_mark(c, 0, stream);
         st = launch_gemm_select(c, qsrc, qld, batch_max, count_dev, stream);
         if (st != FI_OK) return st;
+        prof_mark(c, 1, stream);
         fa.parts = -1;
         fa.list_len = -1;
         fa.refine = 1;
@@ -216,7 +232,7 @@ fi_status_t fi_cache_create(const fi_cache_config_t *cfg, fi_cache_t **out) {
     size_t entries = (size_t)16 * c->sm_count * 4 * cfg->k;
     if (entries < (size_t)cfg->max_batch * cfg->k * 2) entries = (size_t)cfg->max_batch * cfg->k * 2;
     if (bf16) {
-        size_t g = gemm_part_entries(cfg->max_batch, cfg->capacity, c->sm_count, cfg->k);
+        size_t g = gemm_part_entries(cfg->max_batch, cfg->capacity, c->sm_count, cfg->k, cfg->dim);
         if (g > entries) entries = g;
     }
     if (st == FI_OK) need(dev_alloc(&c->part_score, entries, "allocating candidate scores"));
@@ -536,6 +552,55 @@ fi_status_t fi_cache_poll_status(fi_cache_t *c) {
         set_error("a kernel gave up on a bounded wait (code %d, site %d)", word & 0xFF, word >> 8);
         return FI_ERR_TIMEOUT;
     }
+    return FI_OK;
+}
+
+fi_status_t fi_cache_set_profiling(fi_cache_t *c, int32_t enable) {
+    if (!c) {
+        set_error("fi_cache_set_profiling: null cache");
+        return FI_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(c->cfg.device);
+    if (enable && !c->prof_ev) {
+        c->prof_ev = new (std::nothrow) cudaEvent_t[2 * kProfSlots];
+        if (!c->prof_ev) {
+            set_error("fi_cache_set_profiling: out of host memory");
+            return FI_ERR_OOM;
+        }
+        for (int i = 0; i < 2 * kProfSlots; ++i) {
+            cudaError_t e = cudaEventCreate(&c->prof_ev[i]);
+            if (e != cudaSuccess) {
+                for (int j = 0; j < i; ++j) cudaEventDestroy(c->prof_ev[j]);
+                delete[] c->prof_ev;
+                c->prof_ev = nullptr;
+                return cuda_fail(e, "fi_cache_set_profiling: creating events");
+            }
+        }
+    }
+    c->prof_on = enable != 0;
+    c->prof_n = 0;
+    return FI_OK;
+}
+
+fi_status_t fi_cache_read_profile(fi_cache_t *c, float *total_ms, int32_t *launches) {
+    if (!c || !total_ms || !launches) {
+        set_error("fi_cache_read_profile: null argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    *total_ms = 0.f;
+    *launches = 0;
+    if (!c->prof_ev) return FI_OK;
+    DeviceGuard guard(c->cfg.device);
+    const int n = c->prof_n < kProfSlots ? c->prof_n : kProfSlots;
+    for (int i = 0; i < n; ++i) {
+        cudaError_t e = cudaEventSynchronize(c->prof_ev[2 * i + 1]);
+        float ms = 0.f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]);
+        if (e != cudaSuccess) return cuda_fail(e, "fi_cache_read_profile: reading events");
+        *total_ms += ms;
+    }
+    *launches = n;
+    c->prof_n = 0;
     return FI_OK;
 }
 

@@ -87,7 +87,6 @@ __global__ void __launch_bounds__(kFinThreads) finalize_kernel(FinalizeParams p)
     __shared__ int32_t cand_i[kMaxK];
     __shared__ float red_s[kFinWarps];
     __shared__ int32_t red_i[kFinWarps];
-    __shared__ int32_t s_cand_n;
 
     const int count = p.count_dev ? min(*p.count_dev, p.batch_max) : p.batch_max;
     const int b = blockIdx.x;

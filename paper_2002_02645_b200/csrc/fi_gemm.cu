@@ -6,9 +6,14 @@
 // accumulator tiles back from TMEM (one query row per thread) and keeps the `list_len` smallest scores of its
 // row in registers.  The exact distances of those few candidates are recomputed afterwards (finalize_kernel).
 //
-// Roles inside a CTA of 192 threads: warp 0 = TMA producer (one lane), warp 1 = TMEM owner and MMA issuer
-// (one lane), warps 2..5 = epilogue.  Shared-memory stages are handed over with mbarriers; the accumulator is
-// double-buffered in TMEM (2 x 256 columns) so the select of one tile overlaps the MMAs of the next.
+// Roles inside a CTA: warp 0 = TMA producer (one lane), warp 1 = TMEM owner and MMA issuer (one lane), the
+// other warps = epilogue, one thread per query row.  Shared-memory stages are handed over with mbarriers.
+// Two tile heights are compiled:
+//   128 queries: accumulator double-buffered in TMEM (2 x 256 columns), so the select of one tile overlaps
+//                the MMAs of the next; 4 epilogue warps.  For short rows (few k-blocks per tile).
+//   256 queries: two 128-row MMAs share every cache-row stage, which halves the bytes the CTA pulls from L2
+//                per flop (the kernel is bound by L2-to-SM bandwidth, not by the tensor pipe); the two
+//                accumulators fill TMEM, so select and MMAs alternate; 8 epilogue warps.  For long rows.
 // Every wait is bounded: a wait that runs out sets the cache's status word and the CTA drains and returns.
 #include <cuda_bf16.h>
 
@@ -19,19 +24,17 @@ namespace fi {
 namespace {
 
 constexpr int kBlockK = 64;                       // bf16 elements per k-block: 128 bytes, one swizzle row
-constexpr int kStages = 4;
+constexpr int kMaxStages = 8;
 constexpr int kMaxTileN = 256;                    // cache rows per tile (MMA N), multiple of 16
 constexpr int kABytes = kTileM * kBlockK * 2;     // 16 KiB
-constexpr int kBBytes = kMaxTileN * kBlockK * 2;  // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kGemmThreads = 192;
-constexpr int kEpiWarps = 4;
+constexpr int kStageRegionBytes = 200 * 1024;     // operand ring; a stage is A (16 or 32 KiB) + B (tile width x 128 bytes)
+constexpr int kMaxEpiWarps = 8;
 constexpr int kTmemCols = 512;
 constexpr uint64_t kWaitLimitNs = 4000000000ull;  // 4 s: far beyond any tile, short enough to get the GPU back
 
 struct __align__(8) SmemCtl {
-    uint64_t full[kStages];
-    uint64_t empty[kStages];
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
@@ -39,8 +42,8 @@ struct __align__(8) SmemCtl {
     GemmPlan plan;
 };
 
-constexpr int kNormSmemBytes = kEpiWarps * 2 * kMaxTileN * 4;   // per epilogue warp, per accumulator buffer
-constexpr int kGemmSmemBytes = 1024 /*alignment slack*/ + kStages * kStageBytes + kNormSmemBytes + (int)sizeof(SmemCtl);
+constexpr int kNormSmemBytes = kMaxEpiWarps * kMaxTileN * 4;   // 4 warps x 2 accumulator buffers, or 8 warps x 1
+constexpr int kGemmSmemBytes = 1024 /*alignment slack*/ + kStageRegionBytes + kNormSmemBytes + (int)sizeof(SmemCtl);
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -198,26 +201,32 @@ struct TileWalk {
     }
 };
 
-template <int KP>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+// MSUB = 128-row MMAs per CTA tile (1 or 2)
+template <int KP, int MSUB>
+__global__ void __launch_bounds__(64 + 128 * MSUB, 1)
 gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_x64,
                    const __grid_constant__ CUtensorMap tmap_x16, const float *__restrict__ norms, long long n_entries,
                    int dim, int batch_max, const int32_t *__restrict__ count_dev, int k,
                    float *__restrict__ part_score, int32_t *__restrict__ part_idx, GemmPlan *__restrict__ plan_out,
                    int32_t *__restrict__ status) {
+    constexpr int kTileRows = kTileM * MSUB;
+    constexpr int kATileBytes = kABytes * MSUB;
+    constexpr int kAccBufs = MSUB == 1 ? 2 : 1;   // accumulator sets in TMEM
+    constexpr int kEpiThreads = 128 * MSUB;
+
     extern __shared__ unsigned char smem_raw[];
     // operand stages need 1024-byte alignment for the 128-byte swizzle
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char *stage_base = smem;
-    float *norm_smem = reinterpret_cast<float *>(smem + kStages * kStageBytes);
-    SmemCtl *ctl = reinterpret_cast<SmemCtl *>(smem + kStages * kStageBytes + kNormSmemBytes);
+    float *norm_smem = reinterpret_cast<float *>(smem + kStageRegionBytes);
+    SmemCtl *ctl = reinterpret_cast<SmemCtl *>(smem + kStageRegionBytes + kNormSmemBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         int count = count_dev ? min(*count_dev, batch_max) : batch_max;
         if (count < 0) count = 0;
-        ctl->plan = make_gemm_plan(count, n_entries, (int)gridDim.x, k);
+        ctl->plan = make_gemm_plan(count, n_entries, (int)gridDim.x, k, kTileRows);
         ctl->abort_flag = 0;
         if (blockIdx.x == 0) *plan_out = ctl->plan;
     }
@@ -230,15 +239,21 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     walk.setup(plan, q, n_entries);
     if (walk.tiles == 0) return;
     const int num_kb = (dim + kBlockK - 1) / kBlockK;
+    // groups in which this CTA has a query tile: a prefix of all groups
+    const int my_groups = m_local < plan.m_tiles ? (plan.m_tiles - m_local + plan.mg - 1) / plan.mg : 0;
+    if (my_groups == 0) return;
+    // as many stages as fit: narrower tiles leave room for a deeper ring
+    const int stage_bytes = kATileBytes + walk.tile_w * (kBlockK * 2);
+    const int num_stages = min(kMaxStages, kStageRegionBytes / stage_bytes);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(&ctl->full[s], 1);
             mbar_init(&ctl->empty[s], 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&ctl->tmem_full[a], 1);
-            mbar_init(&ctl->tmem_empty[a], kEpiWarps * 32);
+            mbar_init(&ctl->tmem_empty[a], kEpiThreads);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -257,39 +272,48 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t it = 0, stage = 0, ph = 0;
             bool ok = true;
-            for (int g = 0; g < plan.groups && ok; ++g) {
+            for (int g = 0; g < my_groups && ok; ++g) {
                 const int m_tile = g * plan.mg + m_local;
-                if (m_tile >= plan.m_tiles) continue;
                 for (int t = 0; t < walk.tiles && ok; ++t) {
                     const int col0 = walk.col0(t), w = walk.width(t);
                     for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                        const int s = it % kStages;
-                        const uint32_t ph = (it / kStages) & 1;
-                        if (!mbar_wait(&ctl->empty[s], ph ^ 1, ctl, status, 1)) {
+                        if (!mbar_wait(&ctl->empty[stage], ph ^ 1, ctl, status, 1)) {
                             ok = false;
                             break;
                         }
-                        mbar_expect_tx(&ctl->full[s], (uint32_t)(kABytes + w * kBlockK * 2));
-                        const uint32_t a_dst = smem_u32(stage_base + s * kStageBytes);
-                        const uint32_t b_dst = a_dst + kABytes;
-                        tma_load_2d(a_dst, &tmap_q, &ctl->full[s], kb * kBlockK, m_tile * kTileM);
+                        mbar_expect_tx(&ctl->full[stage], (uint32_t)(kATileBytes + w * kBlockK * 2));
+                        const uint32_t a_dst = smem_u32(stage_base + stage * stage_bytes);
+                        const uint32_t b_dst = a_dst + kATileBytes;
+#pragma unroll
+                        for (int ms = 0; ms < MSUB; ++ms)
+                            tma_load_2d(a_dst + ms * kABytes, &tmap_q, &ctl->full[stage], kb * kBlockK,
+                                        m_tile * kTileRows + ms * kTileM);
                         int r = 0;
                         for (; r + 64 <= w; r += 64)
-                            tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x64, &ctl->full[s], kb * kBlockK, col0 + r);
+                            tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x64, &ctl->full[stage], kb * kBlockK, col0 + r);
                         for (; r < w; r += 16)
-                            tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x16, &ctl->full[s], kb * kBlockK, col0 + r);
+                            tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x16, &ctl->full[stage], kb * kBlockK, col0 + r);
+                        if (++stage == (uint32_t)num_stages) {
+                            stage = 0;
+                            ph ^= 1;
+                        }
                     }
                 }
             }
             if (!ok) {
                 // gave up: let the copies already issued land before the CTA leaves
-                uint32_t issued = it;
-                uint32_t first = issued > (uint32_t)kStages ? issued - kStages : 0;
-                for (uint32_t j = first; j < issued; ++j) {
+                uint32_t back = it < (uint32_t)num_stages ? it : (uint32_t)num_stages;
+                uint32_t s2 = stage, p2 = ph;
+                for (uint32_t j = 0; j < back; ++j) {
+                    if (s2 == 0) {
+                        s2 = num_stages;
+                        p2 ^= 1;
+                    }
+                    --s2;
                     uint64_t t0 = global_timer_ns();
-                    while (!mbar_try(&ctl->full[j % kStages], (j / kStages) & 1))
+                    while (!mbar_try(&ctl->full[s2], p2))
                         if (global_timer_ns() - t0 > 20000000ull) break;
                 }
             }
@@ -297,14 +321,12 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            uint32_t it = 0, tile_no = 0;
+            uint32_t tile_no = 0, stage = 0, ph = 0;
             bool ok = true;
-            for (int g = 0; g < plan.groups && ok; ++g) {
-                const int m_tile = g * plan.mg + m_local;
-                if (m_tile >= plan.m_tiles) continue;
+            for (int g = 0; g < my_groups && ok; ++g) {
                 for (int t = 0; t < walk.tiles && ok; ++t, ++tile_no) {
                     const int w = walk.width(t);
-                    const uint32_t acc = tile_no & 1, acc_ph = (tile_no >> 1) & 1;
+                    const uint32_t acc = tile_no % kAccBufs, acc_ph = (tile_no / kAccBufs) & 1;
                     if (!mbar_wait(&ctl->tmem_empty[acc], acc_ph ^ 1, ctl, status, 2)) {
                         ok = false;
                         break;
@@ -312,21 +334,26 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + acc * kMaxTileN;
                     const uint32_t idesc = umma_instr_desc(w);
-                    for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                        const int s = it % kStages;
-                        const uint32_t ph = (it / kStages) & 1;
-                        if (!mbar_wait(&ctl->full[s], ph, ctl, status, 3)) {
+                    for (int kb = 0; kb < num_kb; ++kb) {
+                        if (!mbar_wait(&ctl->full[stage], ph, ctl, status, 3)) {
                             ok = false;
                             break;
                         }
                         tc_fence_after();
-                        const uint32_t a_addr = smem_u32(stage_base + s * kStageBytes);
-                        const uint64_t adesc = umma_smem_desc(a_addr);
-                        const uint64_t bdesc = umma_smem_desc(a_addr + kABytes);
+                        const uint32_t a_addr = smem_u32(stage_base + stage * stage_bytes);
+                        const uint64_t bdesc = umma_smem_desc(a_addr + kATileBytes);
 #pragma unroll
-                        for (int kk = 0; kk < kBlockK / 16; ++kk)
-                            umma_bf16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | kk) != 0);
-                        umma_commit(&ctl->empty[s]);   // frees the stage once these MMAs have read it
+                        for (int kk = 0; kk < kBlockK / 16; ++kk) {
+#pragma unroll
+                            for (int ms = 0; ms < MSUB; ++ms)
+                                umma_bf16(d_tmem + ms * kMaxTileN, umma_smem_desc(a_addr + ms * kABytes) + 2 * kk,
+                                          bdesc + 2 * kk, idesc, (kb | kk) != 0);
+                        }
+                        umma_commit(&ctl->empty[stage]);   // frees the stage once these MMAs have read it
+                        if (++stage == (uint32_t)num_stages) {
+                            stage = 0;
+                            ph ^= 1;
+                        }
                     }
                     if (ok) umma_commit(&ctl->tmem_full[acc]);
                 }
@@ -334,20 +361,20 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         }
     } else {
         // ------------------------------------------------------------ epilogue: per-row select
-        const int ew = warp - 2;              // 0..3, staging slot
+        const int ew = warp - 2;              // 0 .. 4*MSUB-1
+        const int msub = ew >> 2;             // which 128-row MMA this warp drains
         const int quarter = warp & 3;         // TMEM lanes this warp may read: 32*quarter .. +31
-        const int row_in_tile = quarter * 32 + lane;
-        float *my_norm = norm_smem + ew * (2 * kMaxTileN);
+        const int row_in_tile = msub * kTileM + quarter * 32 + lane;
+        float *my_norm = norm_smem + ew * (kAccBufs * kMaxTileN);
         TopList<KP> top;
         uint32_t tile_no = 0;
         bool ok = true;
-        for (int g = 0; g < plan.groups && ok; ++g) {
+        for (int g = 0; g < my_groups && ok; ++g) {
             const int m_tile = g * plan.mg + m_local;
-            if (m_tile >= plan.m_tiles) continue;
             top.reset();
             for (int t = 0; t < walk.tiles && ok; ++t, ++tile_no) {
                 const int col0 = walk.col0(t), w = walk.width(t);
-                const uint32_t acc = tile_no & 1, acc_ph = (tile_no >> 1) & 1;
+                const uint32_t acc = tile_no % kAccBufs, acc_ph = (tile_no / kAccBufs) & 1;
                 float *nrm = my_norm + acc * kMaxTileN;
                 // squared norms of this tile's cache rows; rows past the end get +inf and never enter a list
                 for (int c = lane; c < w; c += 32)
@@ -357,7 +384,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, status, 4));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kMaxTileN;
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (acc + msub) * kMaxTileN;
                 for (int c0 = 0; c0 < w; c0 += 16) {
                     uint32_t v[16];
                     __syncwarp();
@@ -374,7 +401,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 __syncwarp();
             }
             if (ok) {
-                const int row = m_tile * kTileM + row_in_tile;
+                const int row = m_tile * kTileRows + row_in_tile;
                 if (row < plan.count) {
                     const long long o = ((long long)row * plan.parts + q) * KP;
 #pragma unroll
@@ -433,10 +460,10 @@ fi_status_t encode_bf16_map(CUtensorMap *map, const void *base, uint64_t rows, u
     return FI_OK;
 }
 
-template <int KP>
+template <int KP, int MSUB>
 fi_status_t launch_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, const int32_t *count_dev, cudaStream_t stream) {
     static bool attr_set = false;
-    auto kern = gemm_select_kernel<KP>;
+    auto kern = gemm_select_kernel<KP, MSUB>;
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) != cudaSuccess) {
             set_error("cannot reserve %d bytes of shared memory for the distance GEMM", kGemmSmemBytes);
@@ -445,15 +472,29 @@ fi_status_t launch_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, con
         }
         attr_set = true;
     }
-    kern<<<c->sm_count, kGemmThreads, kGemmSmemBytes, stream>>>(tq, c->tmap_rows64, c->tmap_rows16, c->norms,
-                                                               (long long)c->size, c->cfg.dim, batch_max, count_dev,
-                                                               c->cfg.k, c->part_score, c->part_idx, c->plan_dev,
-                                                               c->status_dev);
+    kern<<<c->sm_count, 64 + 128 * MSUB, kGemmSmemBytes, stream>>>(tq, c->tmap_rows64, c->tmap_rows16, c->norms,
+                                                                  (long long)c->size, c->cfg.dim, batch_max, count_dev,
+                                                                  c->cfg.k, c->part_score, c->part_idx, c->plan_dev,
+                                                                  c->status_dev);
     count_launch();
     return check_launch("gemm_select_kernel");
 }
 
+template <int MSUB>
+fi_status_t launch_msub(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, const int32_t *count_dev, cudaStream_t stream) {
+    switch (gemm_list_len(c->cfg.k)) {
+        case 4: return launch_kp<4, MSUB>(c, tq, batch_max, count_dev, stream);
+        case 8: return launch_kp<8, MSUB>(c, tq, batch_max, count_dev, stream);
+        case 16: return launch_kp<16, MSUB>(c, tq, batch_max, count_dev, stream);
+        default: return launch_kp<32, MSUB>(c, tq, batch_max, count_dev, stream);
+    }
+}
+
 }  // namespace
+
+// Query rows per CTA tile: 256 when the batch can fill it and a tile's k-loop is long enough (>= 32 k-blocks) to
+// dwarf the select that can no longer overlap it; 128 otherwise.
+int gemm_tile_m(int batch_max, int dim) { return (batch_max > kTileM && dim >= 32 * kBlockK) ? 2 * kTileM : kTileM; }
 
 fi_status_t ensure_tensor_maps(fi_cache *c) {
     if (c->tmaps_ready) return FI_OK;
@@ -465,12 +506,13 @@ fi_status_t ensure_tensor_maps(fi_cache *c) {
     return FI_OK;
 }
 
-size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k) {
+size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, int dim) {
     size_t worst = 0;
-    int m_tiles_max = (max_batch + kTileM - 1) / kTileM;
+    const int tile_m = gemm_tile_m(max_batch, dim);
+    int m_tiles_max = (max_batch + tile_m - 1) / tile_m;
     for (int mt = 1; mt <= m_tiles_max; ++mt) {
-        GemmPlan p = make_gemm_plan(mt * kTileM, capacity, sm_count, k);
-        size_t e = (size_t)mt * kTileM * (size_t)p.parts * (size_t)p.list_len;
+        GemmPlan p = make_gemm_plan(mt * tile_m, capacity, sm_count, k, tile_m);
+        size_t e = (size_t)mt * tile_m * (size_t)p.parts * (size_t)p.list_len;
         if (e > worst) worst = e;
     }
     return worst;
@@ -492,12 +534,8 @@ fi_status_t launch_gemm_select(fi_cache *c, const void *queries_compact, int64_t
     CUtensorMap tq;
     st = encode_bf16_map(&tq, queries_compact, (uint64_t)batch_max, (uint64_t)c->cfg.dim, (uint64_t)ld_elems, kTileM);
     if (st != FI_OK) return st;
-    switch (gemm_list_len(c->cfg.k)) {
-        case 4: return launch_kp<4>(c, tq, batch_max, count_dev, stream);
-        case 8: return launch_kp<8>(c, tq, batch_max, count_dev, stream);
-        case 16: return launch_kp<16>(c, tq, batch_max, count_dev, stream);
-        default: return launch_kp<32>(c, tq, batch_max, count_dev, stream);
-    }
+    if (gemm_tile_m(batch_max, c->cfg.dim) == kTileM) return launch_msub<1>(c, tq, batch_max, count_dev, stream);
+    return launch_msub<2>(c, tq, batch_max, count_dev, stream);
 }
 
 }  // namespace fi

@@ -11,7 +11,8 @@ namespace fi {
 
 constexpr int kMaxK = 32;          // largest k of a look-up
 constexpr int kStreamMaxBatch = 4; // batches up to this size take the streaming kernel under FI_PATH_AUTO
-constexpr int kTileM = 128;        // queries per GEMM tile (= TMEM lanes)
+constexpr int kTileM = 128;        // queries per MMA (= TMEM lanes); a CTA tile holds 128 or 256 queries
+constexpr int kProfSlots = 256;    // look-ups whose distance-kernel time is kept
 
 // Candidates kept per query by the GEMM path before the exact re-ranking: k plus a margin of 3,
 // rounded up to a list length the select kernel is compiled for.
@@ -20,27 +21,27 @@ __host__ __device__ inline int gemm_list_len(int k) {
     return want <= 4 ? 4 : want <= 8 ? 8 : want <= 16 ? 16 : 32;
 }
 
-// How the tiles of the distance GEMM are spread over the CTAs.  Query tiles (128 rows each) are taken in
-// groups of `mg`; inside a group, CTA (m_local, q) owns query tile m_local and the q-th of `parts` equal
+// How the tiles of the distance GEMM are spread over the CTAs.  Query tiles (`tile_m` = 128 or 256 rows each) are
+// taken in groups of `mg`; inside a group, CTA (m_local, q) owns query tile m_local and the q-th of `parts` equal
 // ranges of cache rows, so CTAs with the same q stream the same cache rows at the same time (they meet in
 // L2) and each query row ends up with `parts` candidate lists.
 struct GemmPlan {
     int32_t count;      // actual batch
-    int32_t m_tiles;    // ceil(count / 128)
+    int32_t m_tiles;    // ceil(count / tile_m)
     int32_t mg;         // query tiles per group
     int32_t groups;     // ceil(m_tiles / mg)
     int32_t parts;      // cache-row ranges per query tile = candidate lists per query
     int32_t range16;    // rows per range, in units of 16 (the last range may be shorter)
     int32_t list_len;   // entries per candidate list
-    int32_t pad;
+    int32_t tile_m;     // query rows per CTA tile
 };
 
-__host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entries, int num_ctas, int k) {
+__host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entries, int num_ctas, int k, int tile_m) {
     GemmPlan p;
     p.count = count;
-    p.m_tiles = (count + kTileM - 1) / kTileM;
+    p.m_tiles = (count + tile_m - 1) / tile_m;
     p.list_len = gemm_list_len(k);
-    p.pad = 0;
+    p.tile_m = tile_m;
     long long n16 = (n_entries + 15) / 16;
     if (p.m_tiles <= 0 || n16 <= 0) {
         p.mg = p.groups = p.parts = 1;
@@ -111,6 +112,10 @@ struct fi_cache {
     CUtensorMap tmap_rows64;
     CUtensorMap tmap_rows16;
     bool tmaps_ready;
+    // optional device timing of the distance kernel
+    bool prof_on;
+    int prof_n;              // look-ups recorded since the last read
+    cudaEvent_t *prof_ev;    // 2 * kProfSlots events, created on first use
 };
 
 namespace fi {
@@ -152,6 +157,7 @@ fi_status_t launch_compact(const fi_cache *c, const fi_cascade_state_t &st, cuda
 fi_status_t launch_cascade_init(const fi_cascade_state_t &st, int32_t num_stages, cudaStream_t stream);
 
 fi_status_t ensure_tensor_maps(fi_cache *c);
-size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k);
+size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, int dim);
+int gemm_tile_m(int batch_max, int dim);
 
 }  // namespace fi

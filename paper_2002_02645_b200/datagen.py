@@ -151,16 +151,19 @@ class Workload:
 
 def make_stage(*, n_cache: int, n_query: int, n_calib: int, dim: int, num_classes: int, dtype: str, kind: str,
                scale: float, seed: int, stage: int, probs: np.ndarray,
-               query_classes: Optional[np.ndarray] = None, calib_classes: Optional[np.ndarray] = None):
+               query_classes: Optional[np.ndarray] = None, calib_classes: Optional[np.ndarray] = None,
+               query_seed: Optional[int] = None):
+    """`query_seed` (default: `seed`) draws another batch of requests against the same cache."""
+    qseed = seed if query_seed is None else query_seed
     means = class_means(num_classes, dim, seed, stage)
     cache_labels = draw_labels(n_cache, probs, seed, _S_CACHE_LABELS, stage)
     cache = _alloc(n_cache, dim, dtype)
     _fill_rows(cache, cache_labels, means, kind=kind, scale=scale, seed=seed, stream=_S_CACHE_NOISE,
                stage=stage, dtype=dtype)
     if query_classes is None:
-        query_classes = draw_labels(n_query, probs, seed, _S_QUERY_LABELS, 0)
+        query_classes = draw_labels(n_query, probs, qseed, _S_QUERY_LABELS, 0)
     queries = _alloc(n_query, dim, dtype)
-    _fill_rows(queries, query_classes, means, kind=kind, scale=scale, seed=seed, stream=_S_QUERY_NOISE,
+    _fill_rows(queries, query_classes, means, kind=kind, scale=scale, seed=qseed, stream=_S_QUERY_NOISE,
                stage=stage, dtype=dtype)
     calib = None
     if n_calib > 0:
@@ -173,11 +176,13 @@ def make_stage(*, n_cache: int, n_query: int, n_calib: int, dim: int, num_classe
 
 
 def single_layer(*, name: str, n_cache: int, n_query: int, dim: int, num_classes: int, dtype: str, sigma: float,
-                 k: int, seed: int = 0, n_copies: int = 0, n_calib: int = 0, zipf: Optional[float] = None) -> Workload:
+                 k: int, seed: int = 0, n_copies: int = 0, n_calib: int = 0, zipf: Optional[float] = None,
+                 query_seed: Optional[int] = None) -> Workload:
     """One cache of ReLU'd Gaussian-mixture vectors; optional exact copies of cache rows among the queries."""
     probs = class_probs(num_classes, zipf)
     st, qc, cc = make_stage(n_cache=n_cache, n_query=n_query, n_calib=n_calib, dim=dim, num_classes=num_classes,
-                            dtype=dtype, kind="relu_mixture", scale=sigma, seed=seed, stage=0, probs=probs)
+                            dtype=dtype, kind="relu_mixture", scale=sigma, seed=seed, stage=0, probs=probs,
+                            query_seed=query_seed)
     meta: Dict[str, object] = {}
     if n_copies > 0:
         g = _rng(seed, _S_COPIES)
@@ -193,7 +198,8 @@ def single_layer(*, name: str, n_cache: int, n_query: int, dim: int, num_classes
 
 
 def cascade(*, name: str, dims: List[int], scales: List[float], kind: str, n_cache: int, n_query: int, n_calib: int,
-            num_classes: int, dtype: str, k: int, seed: int = 0, zipf: Optional[float] = None) -> Workload:
+            num_classes: int, dtype: str, k: int, seed: int = 0, zipf: Optional[float] = None,
+            query_seed: Optional[int] = None) -> Workload:
     """One cache per stage; the class of request r is the same at every stage."""
     probs = class_probs(num_classes, zipf)
     stages: List[StageData] = []
@@ -201,7 +207,7 @@ def cascade(*, name: str, dims: List[int], scales: List[float], kind: str, n_cac
     for s, (dim, scale) in enumerate(zip(dims, scales)):
         st, qc, cc = make_stage(n_cache=n_cache, n_query=n_query, n_calib=n_calib, dim=dim, num_classes=num_classes,
                                 dtype=dtype, kind=kind, scale=scale, seed=seed, stage=s, probs=probs,
-                                query_classes=qc, calib_classes=cc)
+                                query_classes=qc, calib_classes=cc, query_seed=query_seed)
         stages.append(st)
     return Workload(name, num_classes, k, stages, qc, cc, {"scales": list(scales)})
 
@@ -219,38 +225,40 @@ def config1(seed: int = 0) -> Workload:
     return w
 
 
-def config2(seed: int = 0, shrink: int = 1, n_calib: int = 512) -> Workload:
+def config2(seed: int = 0, shrink: int = 1, n_calib: int = 512, query_seed: Optional[int] = None,
+            stages: int = 4) -> Workload:
     """Four-stage ResNet-18/CIFAR-10-shaped cascade, bf16, half-normal values with growing class shifts; k = 5."""
-    dims = [65536 // shrink, 32768 // shrink, 16384 // shrink, 8192 // shrink]
+    dims = [65536 // shrink, 32768 // shrink, 16384 // shrink, 8192 // shrink][:stages]
     w = cascade(name="cfg2_resnet18_cascade" + ("" if shrink == 1 else f"_shrink{shrink}"), dims=dims,
-                scales=[0.2, 0.4, 0.8, 1.6], kind="halfnormal", n_cache=10000 // shrink, n_query=1024 // shrink,
-                n_calib=n_calib // shrink, num_classes=10, dtype="bf16", k=5, seed=seed)
-    w.meta.update(rule="conf_gt", percentiles=[80.0, 60.0, 40.0, 20.0])
+                scales=[0.2, 0.4, 0.8, 1.6][:stages], kind="halfnormal", n_cache=10000 // shrink, n_query=1024 // shrink,
+                n_calib=n_calib // shrink, num_classes=10, dtype="bf16", k=5, seed=seed, query_seed=query_seed)
+    w.meta.update(rule="conf_gt", percentiles=[80.0, 60.0, 40.0, 20.0][:stages])
     return w
 
 
-def config3(seed: int = 0, shrink: int = 1, n_calib: int = 512) -> Workload:
+def config3(seed: int = 0, shrink: int = 1, n_calib: int = 512, query_seed: Optional[int] = None) -> Workload:
     """One layer, 200,000 bf16 entries of 8192 values, sigma 0.7, ReLU; batch 8,192; k = 10."""
     w = single_layer(name="cfg3_large_cache" + ("" if shrink == 1 else f"_shrink{shrink}"), n_cache=200000 // shrink,
                      n_query=8192 // shrink, dim=8192, num_classes=10, dtype="bf16", sigma=0.7, k=10, seed=seed,
-                     n_calib=max(1, n_calib // shrink))
+                     n_calib=max(1, n_calib // shrink), query_seed=query_seed)
     w.meta.update(rule="conf_gt", percentiles=[50.0])
     return w
 
 
-def config4(seed: int = 0, shrink: int = 1, n_calib: int = 512) -> Workload:
+def config4(seed: int = 0, shrink: int = 1, n_calib: int = 512, query_seed: Optional[int] = None) -> Workload:
     """Four-stage ImageNet-shaped cascade: 100,000 entries per stage, 1,000 Zipf(1.1) classes, sigma 0.6; k = 5."""
     w = cascade(name="cfg4_imagenet_cascade" + ("" if shrink == 1 else f"_shrink{shrink}"),
                 dims=[256, 512, 1024, 2048], scales=[0.6] * 4, kind="relu_mixture", n_cache=100000 // shrink,
                 n_query=4096 // shrink, n_calib=max(1, n_calib // shrink), num_classes=1000, dtype="bf16", k=5,
-                seed=seed, zipf=1.1)
+                seed=seed, zipf=1.1, query_seed=query_seed)
     w.meta.update(rule="conf_gt", percentiles=[80.0, 60.0, 40.0, 20.0])
     return w
 
 
-def config5(seed: int = 0, shrink: int = 1, batch: int = 16) -> Workload:
+def config5(seed: int = 0, shrink: int = 1, batch: int = 16, query_seed: Optional[int] = None) -> Workload:
     """Latency regime: 50,000 bf16 entries of 16384 values, sigma 0.5, ReLU; batches of 1, 4, 16; k = 1."""
     w = single_layer(name="cfg5_latency" + ("" if shrink == 1 else f"_shrink{shrink}"), n_cache=50000 // shrink,
-                     n_query=batch, dim=16384, num_classes=10, dtype="bf16", sigma=0.5, k=1, seed=seed)
+                     n_query=batch, dim=16384, num_classes=10, dtype="bf16", sigma=0.5, k=1, seed=seed,
+                     query_seed=query_seed)
     w.meta["rule"] = "dist_le"
     return w
