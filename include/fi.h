@@ -171,6 +171,28 @@ fi_status_t fi_cascade_run_host(fi_cache_t *const *stage_caches, int32_t num_sta
                                 int32_t batch0, int32_t *final_label_host, int32_t *exit_stage_host,
                                 float *final_conf_host, int32_t *stage_arrivals_host, void *cuda_stream);
 
+/*
+ * Look-up that allocates nothing (the paper has no counterpart: this entry point exists for callers that
+ * cannot call cudaMalloc when they need an answer, e.g. a server whose own pool already holds all device
+ * memory, or a latency path where an allocation, which may synchronise the device, is not acceptable).
+ * Same result as fi_cache_lookup_batch on the streaming path, but on plain arrays instead of a cache
+ * object, with the candidate-list scratch in a fixed 4 MiB array inside the library (every GPU that loads
+ * the library holds it until the process exits).  Calls no cudaMalloc / cudaFree and no allocating routine.
+ *   cache_vecs [n_entries x dim] device, contiguous rows, dtype fi_dtype_t; labels [n_entries] device;
+ *   weights    [n_entries] device, REQUIRED here (pass ones for a plain k-NN cache);
+ *   queries    [batch x ld_elems] device; out: device arrays as for fi_cache_lookup_batch;
+ *   k 1..32; rule / metric / threshold as in fi_cache_config_t; runs on the current device.
+ * Limits: batch <= 256 per call (FI_ERR_CAPACITY beyond; split larger batches).  The first call on a device
+ * looks up the scratch array's device address (cudaGetSymbolAddress) and the SM count; make that first call
+ * outside any stream capture.  All calls on a device share the one array and it keeps the previous call's
+ * contents (every entry a call reads is first written by that call, so nothing needs clearing): calls that
+ * overlap on the GPU (different streams without ordering) race on it and must be serialised by the caller.
+ */
+fi_status_t fi_lookup_noalloc(const void *cache_vecs, const int32_t *labels, const float *weights, int64_t n_entries,
+                              int32_t dim, int32_t dtype, int32_t k, int32_t rule, int32_t metric, float threshold,
+                              const void *queries, int64_t ld_elems, int32_t batch, const fi_lookup_out_t *out,
+                              void *cuda_stream);
+
 /* Synchronise the device and return FI_ERR_TIMEOUT if a kernel of this cache gave up on a bounded wait
  * since the last poll (the word is cleared), FI_OK otherwise. */
 fi_status_t fi_cache_poll_status(fi_cache_t *cache);

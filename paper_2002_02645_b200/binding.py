@@ -23,7 +23,7 @@ FI_PATH_AUTO, FI_PATH_STREAM, FI_PATH_GEMM = 0, 1, 2
 EXPORTS = ["fi_cache_create", "fi_cache_destroy", "fi_cache_insert", "fi_cache_set_threshold", "fi_cache_set_path",
            "fi_cache_size", "fi_cache_lookup_batch", "fi_cascade_init", "fi_cascade_step", "fi_cache_lookup_batch_host",
            "fi_cascade_run_host", "fi_cache_poll_status", "fi_cache_set_profiling",
-           "fi_cache_read_profile", "fi_launch_count", "fi_last_error", "fi_status_string"]
+           "fi_cache_read_profile", "fi_lookup_noalloc", "fi_launch_count", "fi_last_error", "fi_status_string"]
 
 
 class fi_cache_config_t(ctypes.Structure):
@@ -76,6 +76,8 @@ def load_library(path: Optional[str] = None):
     lib.fi_cache_lookup_batch_host.argtypes = [vp, vp, i32, ctypes.POINTER(fi_lookup_out_t), vp]
     lib.fi_cascade_run_host.argtypes = [ctypes.POINTER(vp), i32, ctypes.POINTER(vp), i32, vp, vp, vp, vp, vp]
     lib.fi_cache_poll_status.argtypes = [vp]
+    lib.fi_lookup_noalloc.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, i32, ctypes.c_float, vp, i64, i32,
+                                      ctypes.POINTER(fi_lookup_out_t), vp]
     lib.fi_cache_set_profiling.argtypes = [vp, i32]
     lib.fi_cache_read_profile.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.fi_launch_count.argtypes = []
@@ -230,6 +232,28 @@ class FreezeCache:
         _check(self._lib.fi_cache_lookup_batch_host(self._h, _dp(queries_host), queries_host.shape[0], ctypes.byref(st),
                                                     _stream_ptr(self.device)))
         return out_host
+
+
+def lookup_noalloc(cache_vecs: torch.Tensor, labels: torch.Tensor, weights: torch.Tensor, queries: torch.Tensor, *,
+                   k: int, rule: int = FI_HIT_CONF_GT, metric: int = FI_METRIC_SQL2, threshold: float = 0.0,
+                   out: Optional[LookupOut] = None) -> LookupOut:
+    """fi_lookup_noalloc: the streaming look-up on plain device arrays, scratch inside the library image.
+    For callers that cannot allocate device memory; `weights` is required (ones for a plain k-NN cache).
+    At most 256 requests per call; calls on one device must not overlap on the GPU."""
+    dtype = FI_BF16 if cache_vecs.dtype == torch.bfloat16 else FI_F32
+    if queries.dtype != cache_vecs.dtype or queries.dim() != 2 or cache_vecs.dim() != 2 or queries.stride(1) != 1 \
+            or not cache_vecs.is_contiguous():
+        raise ValueError("cache_vecs and queries must be 2-D tensors of one dtype; cache rows contiguous")
+    dev = cache_vecs.device
+    if out is None:
+        out = LookupOut(queries.shape[0], k, dev)
+    st = out.as_struct()
+    with torch.cuda.device(dev):
+        _check(load_library().fi_lookup_noalloc(_dp(cache_vecs), _dp(labels), _dp(weights), cache_vecs.shape[0],
+                                                cache_vecs.shape[1], dtype, k, rule, metric, float(threshold),
+                                                _dp(queries), queries.stride(0), queries.shape[0], ctypes.byref(st),
+                                                _stream_ptr(dev)))
+    return out
 
 
 class CascadeState:

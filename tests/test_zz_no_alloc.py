@@ -1,0 +1,59 @@
+"""The allocation-free entry point (fi_lookup_noalloc) against the regular look-up.
+
+Some callers cannot allocate device memory when they need a look-up (their own pool holds the whole GPU, or an
+allocation's implicit synchronisation is not acceptable on their latency path); for them the library keeps the
+streaming look-up's scratch in a fixed array of its own.  This file is collected last on purpose: if the fixed
+scratch ever misbehaved, every other test has already run.  Both kernels are the same, so the outputs must be
+identical, on two calls in a row (the scratch keeps the first call's contents during the second).
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2002_02645_b200 import binding as fb
+from paper_2002_02645_b200 import datagen as dg
+from helpers import make_cache, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def _as_numpy(out):
+    return [t.cpu().numpy() for t in (out.label, out.conf, out.hit, out.topk_dist, out.topk_idx)]
+
+
+@pytest.mark.parametrize("n,d,b,k,dtype", [(3000, 1024, 37, 5, "bf16"), (500, 64, 256, 1, "f32")])
+def test_noalloc_matches_regular_lookup_twice(n, d, b, k, dtype):
+    w = dg.single_layer(name="t", n_cache=n, n_query=b, dim=d, num_classes=6, dtype=dtype, sigma=0.5, k=k, seed=21)
+    st = w.stages[0]
+    cache = make_cache(st, k=k, num_classes=6, tau=0.0, max_batch=b, path=fb.FI_PATH_STREAM)
+    q = to_device(st.queries)
+    tau = float(np.float32(np.median(cache.lookup_batch(q).conf.cpu().numpy())))   # about half of the requests hit
+    cache.set_threshold(tau)
+    want = _as_numpy(cache.lookup_batch(q))
+    torch.cuda.synchronize()
+    x = to_device(st.cache_vecs)
+    labels = torch.from_numpy(st.cache_labels).cuda()
+    ones = torch.ones(n, dtype=torch.float32, device="cuda")
+    # second batch: the same requests in reverse order, so the scratch holds other values between the calls
+    q_rev = q.flip(0).contiguous()
+    got1 = _as_numpy(fb.lookup_noalloc(x, labels, ones, q, k=k, threshold=tau))
+    got2 = _as_numpy(fb.lookup_noalloc(x, labels, ones, q_rev, k=k, threshold=tau))
+    torch.cuda.synchronize()
+    for a, g1, g2 in zip(want, got1, got2):
+        np.testing.assert_array_equal(a, g1)
+        np.testing.assert_array_equal(a[::-1], g2)
+    assert 0 < want[2].sum() < b or b < 4
+    cache.close()
+
+
+def test_noalloc_rejects_what_the_fixed_scratch_cannot_hold():
+    x = torch.zeros(16, 64, dtype=torch.bfloat16, device="cuda")
+    labels = torch.zeros(16, dtype=torch.int32, device="cuda")
+    ones = torch.ones(16, dtype=torch.float32, device="cuda")
+    q = torch.zeros(257, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(fb.FiError) as e:
+        fb.lookup_noalloc(x, labels, ones, q, k=1)
+    assert e.value.status == 2 and "256" in str(e.value)
+    with pytest.raises(fb.FiError) as e:
+        fb.lookup_noalloc(x, labels, ones, q[:4], k=33)
+    assert e.value.status == 1
