@@ -46,6 +46,25 @@ def load_peaks():
         return dict(FALLBACK_PEAKS), "fallback"
 
 
+def captured_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch of `kernel` on `workload` from the committed ncu summary, or None when there is no
+    capture or the kernel's source has changed since (the line carries the source file's sha256)."""
+    import hashlib
+    src = {"gemm_select_kernel": "fi_gemm.cu", "stream_lookup_kernel": "fi_stream.cu"}.get(kernel)
+    try:
+        with open(os.path.join(ROOT, "paper_2002_02645_b200", "csrc", src), "rb") as f:
+            digest = hashlib.sha256(f.read()).hexdigest()
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) >= 4 and not line.startswith("#") and parts[0] == kernel and parts[1] == workload \
+                        and parts[3] == digest:
+                    return float(parts[2])
+    except Exception:
+        pass
+    return None
+
+
 class ClockSampler:
     """nvidia-smi clocks and throttle reasons, sampled while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -104,14 +123,14 @@ def dist_env():
 
 # ---------------------------------------------------------------------------------------------- workloads
 
-def build_workload(name: str, seed: int, query_seed=None):
+def build_workload(name: str, seed: int, query_seed=None, batch=16):
     from paper_2002_02645_b200 import datagen as dg
     if name == "cfg2":
         return dg.config2(seed=seed, query_seed=query_seed)
     if name == "cfg3":
         return dg.config3(seed=seed, query_seed=query_seed)
     if name == "cfg5":
-        return dg.config5(seed=seed, batch=16, query_seed=query_seed)
+        return dg.config5(seed=seed, batch=batch, query_seed=query_seed)
     if name == "cfg2-small":       # same recipe, 1/16 of the sizes: a quick functional run
         return dg.config2(seed=seed, shrink=16, query_seed=query_seed)
     if name == "cfg2-s0":          # first stage of cfg2 alone (10,000 x 65536, batch 1,024): the dominant GEMM
@@ -172,7 +191,8 @@ def run_ours(args):
 
     t_gen = time.time()
     # every rank serves its own requests: same caches, batch drawn from the rank's own seed
-    w = build_workload(args.workload, seed=0, query_seed=None if (rank == 0 or args.same_batch) else 1000 + rank)
+    w = build_workload(args.workload, seed=0, query_seed=None if (rank == 0 or args.same_batch) else 1000 + rank,
+                       batch=args.batch)
     t_gen = time.time() - t_gen
 
     n_stage = len(w.stages)
@@ -263,6 +283,21 @@ def run_ours(args):
     ms_per_step = ms_total / args.steps
     value = world * b0 * args.steps / (ms_total * 1e-3)
 
+    # ---- per-look-up device latency (latency workload): every look-up between its own pair of events
+    latency = None
+    if args.workload == "cfg5":
+        n_lat = max(1000, args.steps)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_lat)]
+        fence()
+        for e0, e1 in evs:
+            e0.record()
+            step()
+            e1.record()
+        fence()
+        lat = sorted(e0.elapsed_time(e1) * 1e3 for e0, e1 in evs)
+        latency = {"lookups": n_lat, "p50_us": lat[len(lat) // 2], "p99_us": lat[int(len(lat) * 0.99)],
+                   "min_us": lat[0], "max_us": lat[-1]}
+
     # ---- end to end through the host-buffer entry point
     host_acts = [to_pinned(st.queries) for st in w.stages]
     h_label = torch.empty(b0, dtype=torch.int32).pin_memory()
@@ -304,20 +339,24 @@ def run_ours(args):
     roofline = None
     if n_launch0 > 0 and ms0 > 0:
         avg_s = ms0 / n_launch0 * 1e-3
-        if b0 > 4:
-            flops = 2.0 * b0 * n0 * d0
+        flops = 2.0 * b0 * n0 * d0
+        nbytes = n0 * d0 * st0.cache_vecs.itemsize + b0 * d0 * st0.cache_vecs.itemsize + 4.0 * n0
+        gemm = st0.dtype == "bf16" and b0 > 4
+        kernel = "gemm_select_kernel" if gemm else "stream_lookup_kernel"
+        # the slower of the flops at the tensor peak and the bytes at the copy bandwidth bounds the launch
+        tensor_bound = gemm and flops / (peaks["bf16_tflops"] * 1e12) > nbytes / (peaks["hbm_gbs"] * 1e9)
+        if tensor_bound:
             achieved = flops / avg_s / 1e12
-            roofline = {"bound": "tensor", "kernel": "gemm_select_kernel (stage 0)", "achieved": achieved,
+            roofline = {"bound": "tensor", "kernel": kernel + " (stage 0)", "achieved": achieved,
                         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
-                        "peak_source": f"bf16 burst, {peak_src}", "traffic": None,
-                        "avg_launch_ms": avg_s * 1e3, "launches": n_launch0}
+                        "peak_source": f"cuBLAS bf16 burst, {peak_src} (timed region well under a second)"}
         else:
-            nbytes = n0 * d0 * 2.0 + b0 * d0 * 2.0
             achieved = nbytes / avg_s / 1e9
-            roofline = {"bound": "hbm", "kernel": "stream_lookup_kernel", "achieved": achieved,
+            roofline = {"bound": "hbm", "kernel": kernel + " (stage 0)", "achieved": achieved,
                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                        "peak_source": f"copy bandwidth, {peak_src}", "traffic": None,
-                        "avg_launch_ms": avg_s * 1e3, "launches": n_launch0}
+                        "peak_source": f"copy bandwidth, {peak_src}"}
+        roofline.update({"traffic": captured_traffic(kernel, w.name), "avg_launch_ms": avg_s * 1e3,
+                         "launches": n_launch0, "algorithmic_flops": flops, "algorithmic_bytes": nbytes})
     stage_info = []
     for l, (ms_l, n_l) in enumerate(prof):
         if n_l:
@@ -343,6 +382,8 @@ def run_ours(args):
                            "parallelism": f"replicas x{world}", "datagen_s": round(t_gen, 1)},
                 "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
                 "stages": stage_info, "cpu_baseline": cpu_baseline}
+        if latency is not None:
+            line["latency"] = latency
         print(json.dumps(line))
     for c in caches:
         c.close()
@@ -386,7 +427,7 @@ def run_reference(args):
     rank, _, world = dist_env()
     if rank != 0:
         return
-    w = build_workload(args.workload, seed=0)
+    w = build_workload(args.workload, seed=0, batch=args.batch)
     from oracle import fi_oracle as fo
     taus = []
     for s, p in zip(w.stages, w.meta.get("percentiles", [50.0] * len(w.stages))):
@@ -425,6 +466,7 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg5", "cfg2-small", "cfg2-s0"])
     ap.add_argument("--cpu-sample", type=int, default=0,
                     help="requests per oracle timing (0: sized for 10-30 s of CPU work)")
+    ap.add_argument("--batch", type=int, default=16, help="batch of the latency workload (cfg5): 1, 4 or 16")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--same-batch", action="store_true", help="every rank serves the same batch")
     args = ap.parse_args()

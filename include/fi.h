@@ -53,8 +53,8 @@ typedef enum { FI_HIT_CONF_GT = 0, FI_HIT_DIST_LE = 1 } fi_hit_rule_t;
 /* The d_j of the confidence sum (Sec. 3): squared L2 distance, or its square root. */
 typedef enum { FI_METRIC_SQL2 = 0, FI_METRIC_L2 = 1 } fi_metric_t;
 
-/* Which kernels serve a look-up.  AUTO: the streaming kernel for batches of at most 4 and for float32
- * caches, the tensor-core distance GEMM otherwise.  The other two force a path (bf16 only for GEMM). */
+/* Which kernels serve a look-up.  AUTO: the streaming kernel for single requests and for float32 caches,
+ * the tensor-core distance GEMM otherwise (from 2 requests on the streaming kernel is bound by its ALU work).  The other two force a path (bf16 only for GEMM). */
 typedef enum { FI_PATH_AUTO = 0, FI_PATH_STREAM = 1, FI_PATH_GEMM = 2 } fi_path_t;
 
 typedef struct {

@@ -10,7 +10,7 @@
 namespace fi {
 
 constexpr int kMaxK = 32;          // largest k of a look-up
-constexpr int kStreamMaxBatch = 4; // batches up to this size take the streaming kernel under FI_PATH_AUTO
+constexpr int kStreamMaxBatch = 1; // batches up to this size take the streaming kernel under FI_PATH_AUTO (bf16)
 constexpr int kTileM = 128;        // queries per MMA (= TMEM lanes); a CTA tile holds 128 or 256 queries
 constexpr int kProfSlots = 256;    // look-ups whose distance-kernel time is kept
 
