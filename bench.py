@@ -131,6 +131,8 @@ def build_workload(name: str, seed: int, query_seed=None, batch=16):
         return dg.config3(seed=seed, query_seed=query_seed)
     if name == "cfg5":
         return dg.config5(seed=seed, batch=batch, query_seed=query_seed)
+    if name == "cfg4":
+        return dg.config4(seed=seed, query_seed=query_seed)
     if name == "cfg2-small":       # same recipe, 1/16 of the sizes: a quick functional run
         return dg.config2(seed=seed, shrink=16, query_seed=query_seed)
     if name == "cfg2-s0":          # first stage of cfg2 alone (10,000 x 65536, batch 1,024): the dominant GEMM
@@ -175,6 +177,7 @@ def run_ours(args):
 
     from paper_2002_02645_b200 import binding as fb
     from paper_2002_02645_b200 import build as fbuild
+    from paper_2002_02645_b200 import sharding
 
     rank, local, world = dist_env()
     if not torch.cuda.is_available():
@@ -276,12 +279,10 @@ def run_ours(args):
     for c in caches:
         c.set_profiling(False)
         c.poll_status()
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    # whole-job figures: slowest rank's time, all ranks' requests
+    ms_total, served = sharding.reduce_timing(ms_total, b0 * args.steps, dev)
     ms_per_step = ms_total / args.steps
-    value = world * b0 * args.steps / (ms_total * 1e-3)
+    value = served / (ms_total * 1e-3)
 
     # ---- per-look-up device latency (latency workload): every look-up between its own pair of events
     latency = None
@@ -322,13 +323,10 @@ def run_ours(args):
         e2e_step()
     fence()
     e2e_s = time.perf_counter() - t0
-    t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_s = float(t.item())
+    e2e_s, e2e_served = sharding.reduce_timing(e2e_s, b0 * e2e_steps, dev)
     h2d = sum(int(a.numel() * a.element_size()) for a in host_acts)
     d2h = b0 * 12 if cascade else b0 * 9
-    e2e = {"value": world * b0 * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+    e2e = {"value": e2e_served / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": 1e3 * e2e_s / e2e_steps}
 
     # ---- roofline of the dominant kernel: the distance kernel of the first (largest) stage
@@ -463,7 +461,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg5", "cfg2-small", "cfg2-s0"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0"])
     ap.add_argument("--cpu-sample", type=int, default=0,
                     help="requests per oracle timing (0: sized for 10-30 s of CPU work)")
     ap.add_argument("--batch", type=int, default=16, help="batch of the latency workload (cfg5): 1, 4 or 16")

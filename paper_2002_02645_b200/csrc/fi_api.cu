@@ -60,7 +60,15 @@ void free_all(fi_cache *c) {
     cudaFree(c->plan_dev);
     cudaFree(c->status_dev);
     cudaFree(c->h2d_stage);
-    cudaFree(c->casc_buf);
+    if (c->copy_ev) {
+        for (int i = 0; i < kMaxHostStages; ++i) cudaEventDestroy(c->copy_ev[i]);
+        delete[] c->copy_ev;
+        c->copy_ev = nullptr;
+    }
+    if (c->copy_stream) {
+        cudaStreamDestroy(c->copy_stream);
+        c->copy_stream = nullptr;
+    }
     if (c->prof_ev) {
         for (int i = 0; i < 2 * kProfSlots; ++i) cudaEventDestroy(c->prof_ev[i]);
         delete[] c->prof_ev;
@@ -470,9 +478,9 @@ fi_status_t fi_cascade_run_host(fi_cache_t *const *caches, int32_t num_stages, c
     DeviceGuard guard(c0->cfg.device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     // device staging: activations of every stage, then the cascade state
-    size_t act_off[64];
-    if (num_stages > 63) {
-        set_error("fi_cascade_run_host: at most 63 stages");
+    size_t act_off[kMaxHostStages];
+    if (num_stages >= kMaxHostStages) {
+        set_error("fi_cascade_run_host: at most %d stages", kMaxHostStages - 1);
         return FI_ERR_INVALID_ARG;
     }
     size_t total = 0;
@@ -493,6 +501,26 @@ fi_status_t fi_cascade_run_host(fi_cache_t *const *caches, int32_t num_stages, c
         if (e != cudaSuccess) return cuda_fail(e, "fi_cascade_run_host: allocating staging");
         c0->h2d_stage_bytes = total;
     }
+    if (!c0->copy_stream) {
+        cudaError_t e = cudaStreamCreateWithFlags(&c0->copy_stream, cudaStreamNonBlocking);
+        if (e != cudaSuccess) return cuda_fail(e, "fi_cascade_run_host: creating the upload stream");
+    }
+    if (!c0->copy_ev) {
+        c0->copy_ev = new (std::nothrow) cudaEvent_t[kMaxHostStages];
+        if (!c0->copy_ev) {
+            set_error("fi_cascade_run_host: out of host memory");
+            return FI_ERR_OOM;
+        }
+        for (int i = 0; i < kMaxHostStages; ++i) {
+            cudaError_t e = cudaEventCreateWithFlags(&c0->copy_ev[i], cudaEventDisableTiming);
+            if (e != cudaSuccess) {
+                for (int j = 0; j < i; ++j) cudaEventDestroy(c0->copy_ev[j]);
+                delete[] c0->copy_ev;
+                c0->copy_ev = nullptr;
+                return cuda_fail(e, "fi_cascade_run_host: creating events");
+            }
+        }
+    }
     unsigned char *base = static_cast<unsigned char *>(c0->h2d_stage);
     int32_t *ibase = reinterpret_cast<int32_t *>(base + state_off);
     int32_t *idx[2] = {ibase, ibase + nb};
@@ -501,11 +529,21 @@ fi_status_t fi_cascade_run_host(fi_cache_t *const *caches, int32_t num_stages, c
     float *final_conf = reinterpret_cast<float *>(ibase + 4 * nb);
     int32_t *counts = ibase + 5 * nb;   // counts[l] = arrivals at stage l; counts[0] unused (= batch0)
 
-    cudaError_t e = cudaSuccess;
-    for (int l = 0; l < num_stages && e == cudaSuccess; ++l)
+    // Uploads go to their own stream in stage order, so stage l+1 arrives while stage l is looked up.  The
+    // staging area is free: the previous call synchronised before returning.  The upload stream first waits
+    // for whatever the caller already queued on the work stream (it may still be using the staging area).
+    cudaEvent_t start_ev = c0->copy_ev[kMaxHostStages - 1];
+    cudaError_t e = cudaEventRecord(start_ev, stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(c0->copy_stream, start_ev, 0);
+    for (int l = 0; l < num_stages && e == cudaSuccess; ++l) {
         e = cudaMemcpyAsync(base + act_off[l], acts_host[l], (size_t)batch0 * caches[l]->cfg.dim * caches[l]->elem_size,
-                            cudaMemcpyHostToDevice, stream);
-    if (e != cudaSuccess) return cuda_fail(e, "fi_cascade_run_host: copying activations");
+                            cudaMemcpyHostToDevice, c0->copy_stream);
+        if (e == cudaSuccess) e = cudaEventRecord(c0->copy_ev[l], c0->copy_stream);
+    }
+    if (e != cudaSuccess) {
+        cudaStreamSynchronize(c0->copy_stream);
+        return cuda_fail(e, "fi_cascade_run_host: copying activations");
+    }
 
     fi_cascade_state_t st;
     memset(&st, 0, sizeof st);
@@ -514,15 +552,26 @@ fi_status_t fi_cascade_run_host(fi_cache_t *const *caches, int32_t num_stages, c
     st.exit_stage = exit_stage;
     st.final_conf = final_conf;
     fi_status_t rc = fi_cascade_init(&st, num_stages, c0->cfg.device, cuda_stream);
-    if (rc != FI_OK) return rc;
+    if (rc != FI_OK) {
+        cudaStreamSynchronize(c0->copy_stream);
+        return rc;
+    }
     for (int l = 0; l < num_stages; ++l) {
         st.stage = l;
         st.active_idx = l == 0 ? nullptr : idx[(l - 1) & 1];
         st.active_count = l == 0 ? nullptr : counts + l;
         st.miss_idx = idx[l & 1];
         st.miss_count = counts + l + 1;
+        e = cudaStreamWaitEvent(stream, c0->copy_ev[l], 0);
+        if (e != cudaSuccess) {
+            cudaStreamSynchronize(c0->copy_stream);
+            return cuda_fail(e, "fi_cascade_run_host: waiting for an upload");
+        }
         rc = fi_cascade_step(caches[l], base + act_off[l], caches[l]->cfg.dim, &st, cuda_stream);
-        if (rc != FI_OK) return rc;
+        if (rc != FI_OK) {
+            cudaStreamSynchronize(c0->copy_stream);
+            return rc;
+        }
     }
     e = cudaMemcpyAsync(final_label_host, final_label, nb * 4, cudaMemcpyDeviceToHost, stream);
     if (e == cudaSuccess) e = cudaMemcpyAsync(exit_stage_host, exit_stage, nb * 4, cudaMemcpyDeviceToHost, stream);

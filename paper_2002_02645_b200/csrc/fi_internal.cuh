@@ -12,6 +12,7 @@ namespace fi {
 constexpr int kMaxK = 32;          // largest k of a look-up
 constexpr int kStreamMaxBatch = 1; // batches up to this size take the streaming kernel under FI_PATH_AUTO (bf16)
 constexpr int kTileM = 128;        // queries per MMA (= TMEM lanes); a CTA tile holds 128 or 256 queries
+constexpr int kMaxHostStages = 64; // stages a host-driven cascade may have
 constexpr int kProfSlots = 256;    // look-ups whose distance-kernel time is kept
 
 // Candidates kept per query by the GEMM path before the exact re-ranking: k plus a margin of 3,
@@ -106,8 +107,8 @@ struct fi_cache {
     // staging for the host-buffer entry points (allocated on first use)
     void *h2d_stage;
     size_t h2d_stage_bytes;
-    int32_t *casc_buf;       // device arrays of a host-driven cascade
-    size_t casc_buf_batch;
+    cudaStream_t copy_stream;   // host-driven cascade: uploads of later stages run here, beside the look-ups
+    cudaEvent_t *copy_ev;       // one "stage uploaded" event per stage (kMaxHostStages), created on first use
     // tensor maps over the cache rows (bf16 only): boxes of 64 and of 16 rows by 64 elements
     CUtensorMap tmap_rows64;
     CUtensorMap tmap_rows16;
