@@ -133,6 +133,10 @@ def build_workload(name: str, seed: int, query_seed=None, batch=16):
         return dg.config5(seed=seed, batch=batch, query_seed=query_seed)
     if name == "cfg4":
         return dg.config4(seed=seed, query_seed=query_seed)
+    if name == "cfg4-s0":          # first stage of cfg4 alone (100,000 x 256, batch 4,096): the select-bound case
+        w = dg.config4(seed=seed, query_seed=query_seed, stages=1)
+        w.name = "cfg4_stage0_only"
+        return w
     if name == "cfg2-small":       # same recipe, 1/16 of the sizes: a quick functional run
         return dg.config2(seed=seed, shrink=16, query_seed=query_seed)
     if name == "cfg2-s0":          # first stage of cfg2 alone (10,000 x 65536, batch 1,024): the dominant GEMM
@@ -461,7 +465,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0"])
     ap.add_argument("--cpu-sample", type=int, default=0,
                     help="requests per oracle timing (0: sized for 10-30 s of CPU work)")
     ap.add_argument("--batch", type=int, default=16, help="batch of the latency workload (cfg5): 1, 4 or 16")

@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(kFinThreads) finalize_kernel(FinalizeParams p)
     const int b = blockIdx.x;
     if (b >= count) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int parts = p.plan ? p.plan->parts : p.parts;
+    const int parts = p.plan ? p.plan->lists : p.parts;
     const int list_len = p.plan ? p.plan->list_len : p.list_len;
     const int entries = parts * list_len;
     const float *ps = p.part_score + (int64_t)b * entries;

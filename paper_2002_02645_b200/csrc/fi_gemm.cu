@@ -6,14 +6,19 @@
 // accumulator tiles back from TMEM (one query row per thread) and keeps the `list_len` smallest scores of its
 // row in registers.  The exact distances of those few candidates are recomputed afterwards (finalize_kernel).
 //
-// Roles inside a CTA: warp 0 = TMA producer (one lane), warp 1 = TMEM owner and MMA issuer (one lane), the
-// other warps = epilogue, one thread per query row.  Shared-memory stages are handed over with mbarriers.
-// Two tile heights are compiled:
+// Roles inside a CTA of 320 threads: warp 0 = TMA producer (one lane), warp 1 = TMEM owner and MMA issuer (one
+// lane), warps 2..9 = epilogue.  Shared-memory stages are handed over with mbarriers.  Two tile heights:
 //   128 queries: accumulator double-buffered in TMEM (2 x 256 columns), so the select of one tile overlaps
-//                the MMAs of the next; 4 epilogue warps.  For short rows (few k-blocks per tile).
+//                the MMAs of the next; two epilogue warps per 32 rows, each taking every other 16-column chunk
+//                and keeping its own list.  For short rows (few k-blocks per tile), where the select dominates.
 //   256 queries: two 128-row MMAs share every cache-row stage, which halves the bytes the CTA pulls from L2
 //                per flop (the kernel is bound by L2-to-SM bandwidth, not by the tensor pipe); the two
-//                accumulators fill TMEM, so select and MMAs alternate; 8 epilogue warps.  For long rows.
+//                accumulators fill TMEM, so select and MMAs alternate; one epilogue warp per 32 rows.
+// Select: a thread owns one query row.  Scores of a 16-column chunk are formed with independent FMAs and
+// tested against the row's current k-th best through one min-tree; the few that pass are parked in a small
+// per-thread queue in shared memory and inserted into the sorted register list once per tile, when all lanes
+// of the warp insert together (inserting on the spot makes the whole warp walk the insert code whenever any
+// one lane has a hit, which made the select 20x slower than the MMAs on short rows).
 // Every wait is bounded: a wait that runs out sets the cache's status word and the CTA drains and returns.
 #include <cuda_bf16.h>
 
@@ -30,7 +35,7 @@ constexpr int kABytes = kTileM * kBlockK * 2;     // 16 KiB
 constexpr int kStageRegionBytes = 200 * 1024;     // operand ring; a stage is A (16 or 32 KiB) + B (tile width x 128 bytes)
 constexpr int kMaxEpiWarps = 8;
 constexpr int kTmemCols = 512;
-constexpr uint64_t kWaitLimitNs = 4000000000ull;  // 4 s: far beyond any tile, short enough to get the GPU back
+constexpr long long kWaitLimitCycles = 8000000000ll;  // about 4 s of SM clocks: far beyond any tile, short enough to get the GPU back
 
 struct __align__(8) SmemCtl {
     uint64_t full[kMaxStages];
@@ -42,16 +47,15 @@ struct __align__(8) SmemCtl {
     GemmPlan plan;
 };
 
-constexpr int kNormSmemBytes = kMaxEpiWarps * kMaxTileN * 4;   // 4 warps x 2 accumulator buffers, or 8 warps x 1
-constexpr int kGemmSmemBytes = 1024 /*alignment slack*/ + kStageRegionBytes + kNormSmemBytes + (int)sizeof(SmemCtl);
+constexpr int kEpiThreads = kMaxEpiWarps * 32;
+constexpr int kGemmThreads = 64 + kEpiThreads;
+constexpr int kNormSmemBytes = kMaxEpiWarps * kMaxTileN * 4;   // 256 floats per epilogue warp
+constexpr int kQueueCap = 8;                                    // pending candidates per epilogue thread
+constexpr int kQueueSmemBytes = kQueueCap * kEpiThreads * 8;    // scores + indices
+constexpr int kGemmSmemBytes =
+    1024 /*alignment slack*/ + kStageRegionBytes + kNormSmemBytes + kQueueSmemBytes + (int)sizeof(SmemCtl);
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ uint64_t global_timer_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
 
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
@@ -79,13 +83,14 @@ __device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity) {
 // another thread of the CTA has already given up.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, SmemCtl *ctl, int32_t *status, int where) {
     if (mbar_try(bar, parity)) return true;
-    uint64_t t0 = global_timer_ns();
+    // the SM's own cycle counter is a register read; the wait sits on the hand-over path of every stage and tile
+    const long long t0 = clock64();
     uint32_t spins = 0;
     while (true) {
         if (mbar_try(bar, parity)) return true;
-        if ((++spins & 0x3FF) == 0) {
+        if ((++spins & 0xFF) == 0) {
             if (ctl->abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            if (clock64() - t0 > kWaitLimitCycles) {
                 ctl->abort_flag = 1;
                 atomicCAS(status, 0, (int32_t)(FI_ERR_TIMEOUT | (where << 8)));
                 return false;
@@ -150,6 +155,13 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[16]) {
                  : "memory");
 }
 
+// order-preserving integer image of a float, so that atomicMin on the image is a float minimum
+__device__ __forceinline__ int32_t float_key(float f) {
+    const int32_t b = __float_as_int(f);
+    return b >= 0 ? b : b ^ 0x7FFFFFFF;
+}
+__device__ __forceinline__ float key_float(int32_t k) { return __int_as_float(k >= 0 ? k : k ^ 0x7FFFFFFF); }
+
 template <int KP>
 struct TopList {
     float s[KP];
@@ -203,23 +215,24 @@ struct TileWalk {
 
 // MSUB = 128-row MMAs per CTA tile (1 or 2)
 template <int KP, int MSUB>
-__global__ void __launch_bounds__(64 + 128 * MSUB, 1)
+__global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_x64,
                    const __grid_constant__ CUtensorMap tmap_x16, const float *__restrict__ norms, long long n_entries,
                    int dim, int batch_max, const int32_t *__restrict__ count_dev, int k,
                    float *__restrict__ part_score, int32_t *__restrict__ part_idx, GemmPlan *__restrict__ plan_out,
-                   int32_t *__restrict__ status) {
+                   int32_t *row_bound, int32_t *__restrict__ status) {
     constexpr int kTileRows = kTileM * MSUB;
     constexpr int kATileBytes = kABytes * MSUB;
     constexpr int kAccBufs = MSUB == 1 ? 2 : 1;   // accumulator sets in TMEM
-    constexpr int kEpiThreads = 128 * MSUB;
 
     extern __shared__ unsigned char smem_raw[];
     // operand stages need 1024-byte alignment for the 128-byte swizzle
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char *stage_base = smem;
     float *norm_smem = reinterpret_cast<float *>(smem + kStageRegionBytes);
-    SmemCtl *ctl = reinterpret_cast<SmemCtl *>(smem + kStageRegionBytes + kNormSmemBytes);
+    float *queue_s = reinterpret_cast<float *>(smem + kStageRegionBytes + kNormSmemBytes);
+    int32_t *queue_i = reinterpret_cast<int32_t *>(queue_s + kQueueCap * kEpiThreads);
+    SmemCtl *ctl = reinterpret_cast<SmemCtl *>(smem + kStageRegionBytes + kNormSmemBytes + kQueueSmemBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -312,9 +325,9 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         p2 ^= 1;
                     }
                     --s2;
-                    uint64_t t0 = global_timer_ns();
+                    const long long t0 = clock64();
                     while (!mbar_try(&ctl->full[s2], p2))
-                        if (global_timer_ns() - t0 > 20000000ull) break;
+                        if (clock64() - t0 > 40000000ll) break;
                 }
             }
         }
@@ -361,49 +374,140 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         }
     } else {
         // ------------------------------------------------------------ epilogue: per-row select
-        const int ew = warp - 2;              // 0 .. 4*MSUB-1
-        const int msub = ew >> 2;             // which 128-row MMA this warp drains
-        const int quarter = warp & 3;         // TMEM lanes this warp may read: 32*quarter .. +31
+        const int ew = warp - 2;                          // 0..7
+        const int quarter = warp & 3;                     // TMEM lanes this warp may read: 32*quarter .. +31
+        const int msub = MSUB == 2 ? (ew >> 2) : 0;       // which 128-row MMA this warp drains
+        const int half = MSUB == 1 ? (ew >> 2) : 0;       // 128-row tiles: which 16-column chunks (even / odd)
+        constexpr int kStep = MSUB == 1 ? 32 : 16;        // distance between this warp's chunks
+        const int first = half * 16;
         const int row_in_tile = msub * kTileM + quarter * 32 + lane;
-        float *my_norm = norm_smem + ew * (kAccBufs * kMaxTileN);
+        const int te = threadIdx.x - 64;                  // 0..255, queue slot
+        float *my_norm = norm_smem + ew * kMaxTileN;      // 256 floats: one buffer (256-row tiles) or two of 128
+        float *qs = queue_s + te;
+        int32_t *qi = queue_i + te;
         TopList<KP> top;
         uint32_t tile_no = 0;
         bool ok = true;
+
+        // Bound shared by every CTA that scans cache rows for the same query: each list publishes its list_len-th
+        // best score, the minimum over lists bounds the list_len-th best of the whole cache from above, and a
+        // score above it can be skipped by every list.  Scores equal to the bound are kept, so which candidates
+        // reach the final merge never depends on the order in which CTAs publish.
+        float bound = __int_as_float(0x7F800000);
+
+        // insert the first n queued candidates of every lane, all lanes together
+        auto flush = [&](int n) {
+            const int rounds = __reduce_max_sync(0xFFFFFFFFu, n);
+            for (int r = 0; r < rounds; ++r) {
+                if (r < n) {
+                    const float sc = qs[r * kEpiThreads];
+                    if (sc < top.s[KP - 1] && sc <= bound) top.insert(sc, qi[r * kEpiThreads]);
+                }
+            }
+        };
+
         for (int g = 0; g < my_groups && ok; ++g) {
             const int m_tile = g * plan.mg + m_local;
+            int32_t *my_bound = row_bound + m_tile * kTileRows + row_in_tile;
             top.reset();
             for (int t = 0; t < walk.tiles && ok; ++t, ++tile_no) {
                 const int col0 = walk.col0(t), w = walk.width(t);
                 const uint32_t acc = tile_no % kAccBufs, acc_ph = (tile_no / kAccBufs) & 1;
-                float *nrm = my_norm + acc * kMaxTileN;
-                // squared norms of this tile's cache rows; rows past the end get +inf and never enter a list
-                for (int c = lane; c < w; c += 32)
-                    nrm[c] = (long long)(col0 + c) < n_entries ? __ldg(norms + col0 + c) : __int_as_float(0x7F800000);
+                float *nrm = my_norm + acc * (kMaxTileN / 2);   // acc is 0 for 256-row tiles
+                int32_t bound_key;   // read past L1: other SMs lower it
+                asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(bound_key) : "l"(my_bound) : "memory");
+                // squared norms of this warp's columns, chunk after chunk; rows past the end of the cache get +inf
+                // and never enter a list
+                for (int li = lane;; li += 32) {
+                    const int c = first + (li >> 4) * kStep + (li & 15);
+                    if (c - (li & 15) >= w) break;
+                    nrm[li] = (long long)(col0 + c) < n_entries ? __ldg(norms + col0 + c) : __int_as_float(0x7F800000);
+                }
                 __syncwarp();
                 // the whole warp takes the same decision, so its lanes stay together for the TMEM loads
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, status, 4));
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (acc + msub) * kMaxTileN;
-                for (int c0 = 0; c0 < w; c0 += 16) {
-                    uint32_t v[16];
-                    __syncwarp();
-                    tmem_ld16(taddr + c0, v);
-                    tmem_ld_wait(v);
+                bound = key_float(bound_key);
+                float thr = fminf(top.s[KP - 1], bound);   // pre-filter: nothing above it can enter the list
+                int cnt = 0;
+
+                auto process = [&](const uint32_t (&v)[16], int c0, int li0) {
+                    const float4 *n4 = reinterpret_cast<const float4 *>(nrm + li0);
+                    const float4 na = n4[0], nb = n4[1], nc = n4[2], nd = n4[3];
+                    const float nv[16] = {na.x, na.y, na.z, na.w, nb.x, nb.y, nb.z, nb.w,
+                                          nc.x, nc.y, nc.z, nc.w, nd.x, nd.y, nd.z, nd.w};
+                    float sc[16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        float sc = fmaf(-2.f, __uint_as_float(v[j]), nrm[c0 + j]);
-                        if (sc < top.s[KP - 1]) top.insert(sc, col0 + c0 + j);
+                    for (int j = 0; j < 16; ++j) sc[j] = fmaf(-2.f, __uint_as_float(v[j]), nv[j]);
+                    float m0 = fminf(fminf(sc[0], sc[1]), fminf(sc[2], sc[3]));
+                    float m1 = fminf(fminf(sc[4], sc[5]), fminf(sc[6], sc[7]));
+                    float m2 = fminf(fminf(sc[8], sc[9]), fminf(sc[10], sc[11]));
+                    float m3 = fminf(fminf(sc[12], sc[13]), fminf(sc[14], sc[15]));
+                    const float mn = fminf(fminf(m0, m1), fminf(m2, m3));
+                    const int cnt0 = cnt;
+                    if (mn <= thr) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            if (sc[j] <= thr) {
+                                if (cnt < kQueueCap) {
+                                    qs[cnt * kEpiThreads] = sc[j];
+                                    qi[cnt * kEpiThreads] = col0 + c0 + j;
+                                }
+                                ++cnt;
+                            }
+                        }
                     }
+                    if (__any_sync(0xFFFFFFFFu, cnt > kQueueCap)) {
+                        // a queue overflowed inside this chunk: insert what was queued before it, then this chunk
+                        // column by column (arrival order, hence the tie order, is kept)
+                        flush(cnt0);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (sc[j] < top.s[KP - 1] && sc[j] <= bound) top.insert(sc[j], col0 + c0 + j);
+                        cnt = 0;
+                        thr = fminf(top.s[KP - 1], bound);
+                    }
+                };
+
+                // two register buffers: the TMEM load of the next chunk is in flight while this one is scanned
+                uint32_t va[16], vb[16];
+                int c0 = first, li0 = 0;
+                if (c0 < w) {
+                    __syncwarp();
+                    tmem_ld16(taddr + c0, va);
+                }
+                while (c0 < w) {
+                    tmem_ld_wait(va);
+                    if (c0 + kStep < w) {
+                        __syncwarp();
+                        tmem_ld16(taddr + c0 + kStep, vb);
+                    }
+                    process(va, c0, li0);
+                    c0 += kStep;
+                    li0 += 16;
+                    if (c0 >= w) break;
+                    tmem_ld_wait(vb);
+                    if (c0 + kStep < w) {
+                        __syncwarp();
+                        tmem_ld16(taddr + c0 + kStep, va);
+                    }
+                    process(vb, c0, li0);
+                    c0 += kStep;
+                    li0 += 16;
                 }
                 tc_fence_before();
                 mbar_arrive(&ctl->tmem_empty[acc]);
+                flush(cnt);   // after the accumulator is released: the MMAs of the next tile can start meanwhile
+                if (top.s[KP - 1] < bound) atomicMin(my_bound, float_key(top.s[KP - 1]));
                 __syncwarp();
             }
             if (ok) {
                 const int row = m_tile * kTileRows + row_in_tile;
                 if (row < plan.count) {
-                    const long long o = ((long long)row * plan.parts + q) * KP;
+                    const int list = MSUB == 1 ? q * 2 + half : q;
+                    const long long o = ((long long)row * plan.lists + list) * KP;
 #pragma unroll
                     for (int e = 0; e < KP; ++e) {
                         part_score[o + e] = top.s[e];
@@ -472,10 +576,16 @@ fi_status_t launch_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, con
         }
         attr_set = true;
     }
-    kern<<<c->sm_count, 64 + 128 * MSUB, kGemmSmemBytes, stream>>>(tq, c->tmap_rows64, c->tmap_rows16, c->norms,
+    // every bound starts at a huge finite value (0x7F7F7F7F as a float is 3.4e38)
+    if (cudaMemsetAsync(c->row_bound, 0x7F, ((size_t)batch_max + 256) * sizeof(int32_t), stream) != cudaSuccess) {
+        set_error("cannot reset the row bounds");
+        cudaGetLastError();
+        return FI_ERR_CUDA;
+    }
+    kern<<<c->sm_count, kGemmThreads, kGemmSmemBytes, stream>>>(tq, c->tmap_rows64, c->tmap_rows16, c->norms,
                                                                   (long long)c->size, c->cfg.dim, batch_max, count_dev,
                                                                   c->cfg.k, c->part_score, c->part_idx, c->plan_dev,
-                                                                  c->status_dev);
+                                                                  c->row_bound, c->status_dev);
     count_launch();
     return check_launch("gemm_select_kernel");
 }
@@ -512,7 +622,7 @@ size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, i
     int m_tiles_max = (max_batch + tile_m - 1) / tile_m;
     for (int mt = 1; mt <= m_tiles_max; ++mt) {
         GemmPlan p = make_gemm_plan(mt * tile_m, capacity, sm_count, k, tile_m);
-        size_t e = (size_t)mt * tile_m * (size_t)p.parts * (size_t)p.list_len;
+        size_t e = (size_t)mt * tile_m * (size_t)p.lists * (size_t)p.list_len;
         if (e > worst) worst = e;
     }
     return worst;

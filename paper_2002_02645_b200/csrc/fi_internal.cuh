@@ -35,6 +35,8 @@ struct GemmPlan {
     int32_t range16;    // rows per range, in units of 16 (the last range may be shorter)
     int32_t list_len;   // entries per candidate list
     int32_t tile_m;     // query rows per CTA tile
+    int32_t lists;      // candidate lists per query = parts x (column halves handled by separate warps)
+    int32_t pad;
 };
 
 __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entries, int num_ctas, int k, int tile_m) {
@@ -43,10 +45,13 @@ __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entrie
     p.m_tiles = (count + tile_m - 1) / tile_m;
     p.list_len = gemm_list_len(k);
     p.tile_m = tile_m;
+    p.pad = 0;
+    p.lists = 0;
     long long n16 = (n_entries + 15) / 16;
     if (p.m_tiles <= 0 || n16 <= 0) {
         p.mg = p.groups = p.parts = 1;
         p.range16 = 0;
+        p.lists = tile_m == kTileM ? 2 : 1;
         return p;
     }
     // pick the group size that needs the fewest MMA columns per CTA in total
@@ -74,6 +79,8 @@ __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entrie
     parts = (n16 + r16 - 1) / r16;   // drop ranges that would be empty
     p.parts = (int32_t)parts;
     p.range16 = (int32_t)r16;
+    // with 128-row tiles two epilogue warps share each row and keep a list each
+    p.lists = p.parts * (tile_m == kTileM ? 2 : 1);
     return p;
 }
 
@@ -102,6 +109,8 @@ struct fi_cache {
     int32_t *slot_label;     // [max_batch] per-slot results of a cascade step
     float *slot_conf;
     uint8_t *slot_hit;
+    int32_t *row_bound;      // [max_batch + 256] per-query upper bound of the list_len-th best score, shared by all
+                             // CTAs of a GEMM launch (order-preserving integer image of the float)
     fi::GemmPlan *plan_dev;  // written by the GEMM kernel, read by the finalize kernel
     int32_t *status_dev;     // device status word (bounded waits that ran out)
     // staging for the host-buffer entry points (allocated on first use)
