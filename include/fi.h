@@ -193,6 +193,19 @@ fi_status_t fi_lookup_noalloc(const void *cache_vecs, const int32_t *labels, con
                               const void *queries, int64_t ld_elems, int32_t batch, const fi_lookup_out_t *out,
                               void *cuda_stream);
 
+/*
+ * ComputeThresholds of Pseudocode 1 for one layer (Sec. 3.1 (ii)): look up n validation activations in the
+ * layer's cache and set THRESHOLDS[layer] to the largest confidence among the look-ups whose label differs from
+ * the label the model itself predicted for that item (0 when no look-up is wrong), "ensuring zero error on the
+ * validation data".  The look-ups run in batches of at most max_batch; the maximum is formed on the device.
+ *   val_acts   [n x ld_elems] device, dtype of the cache; model_labels [n] device int32 (Y[item])
+ *   tau_out    host float, nullable: receives the threshold; wrong_out host int64, nullable: wrong look-ups
+ * The cache's threshold is replaced by the result.  Synchronises the stream before returning.
+ */
+fi_status_t fi_cache_compute_threshold(fi_cache_t *cache, const void *val_acts, int64_t ld_elems,
+                                       const int32_t *model_labels, int64_t n, float *tau_out, int64_t *wrong_out,
+                                       void *cuda_stream);
+
 /* Synchronise the device and return FI_ERR_TIMEOUT if a kernel of this cache gave up on a bounded wait
  * since the last poll (the word is cleared), FI_OK otherwise. */
 fi_status_t fi_cache_poll_status(fi_cache_t *cache);

@@ -142,6 +142,20 @@ def lookup(queries: np.ndarray, cache: np.ndarray, labels: np.ndarray, *, k: int
     return res
 
 
+def compute_threshold(val_queries: np.ndarray, cache: np.ndarray, labels: np.ndarray, model_labels: np.ndarray, *,
+                      k: int, metric: int = METRIC_SQL2, weights: Optional[np.ndarray] = None):
+    """ComputeThresholds of Pseudocode 1 for one layer: walk the validation items in order and raise the
+    threshold to the confidence of every look-up whose label is not the model's (Sec. 3.1 (ii)).  The paper
+    leaves the starting value open; 0 is used.  Returns (threshold, number of wrong look-ups)."""
+    r = lookup(val_queries, cache, labels, k=k, tau=0.0, metric=metric, weights=weights)
+    threshold, wrong = 0.0, 0
+    for item in range(r.label.shape[0]):
+        if int(r.label[item]) != int(model_labels[item]):
+            threshold = max(threshold, float(r.conf[item]))
+            wrong += 1
+    return threshold, wrong
+
+
 def compact(active: np.ndarray, hit: np.ndarray) -> np.ndarray:
     """Ids of `active` whose look-up missed, order kept (Sec. 5, batch reconstruction)."""
     a = np.ascontiguousarray(active, dtype=np.int32)

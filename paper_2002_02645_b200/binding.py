@@ -23,7 +23,7 @@ FI_PATH_AUTO, FI_PATH_STREAM, FI_PATH_GEMM = 0, 1, 2
 EXPORTS = ["fi_cache_create", "fi_cache_destroy", "fi_cache_insert", "fi_cache_set_threshold", "fi_cache_set_path",
            "fi_cache_size", "fi_cache_lookup_batch", "fi_cascade_init", "fi_cascade_step", "fi_cache_lookup_batch_host",
            "fi_cascade_run_host", "fi_cache_poll_status", "fi_cache_set_profiling",
-           "fi_cache_read_profile", "fi_lookup_noalloc", "fi_launch_count", "fi_last_error", "fi_status_string"]
+           "fi_cache_read_profile", "fi_lookup_noalloc", "fi_cache_compute_threshold", "fi_launch_count", "fi_last_error", "fi_status_string"]
 
 
 class fi_cache_config_t(ctypes.Structure):
@@ -76,6 +76,8 @@ def load_library(path: Optional[str] = None):
     lib.fi_cache_lookup_batch_host.argtypes = [vp, vp, i32, ctypes.POINTER(fi_lookup_out_t), vp]
     lib.fi_cascade_run_host.argtypes = [ctypes.POINTER(vp), i32, ctypes.POINTER(vp), i32, vp, vp, vp, vp, vp]
     lib.fi_cache_poll_status.argtypes = [vp]
+    lib.fi_cache_compute_threshold.argtypes = [vp, vp, i64, vp, i64, ctypes.POINTER(ctypes.c_float),
+                                               ctypes.POINTER(i64), vp]
     lib.fi_lookup_noalloc.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, i32, ctypes.c_float, vp, i64, i32,
                                       ctypes.POINTER(fi_lookup_out_t), vp]
     lib.fi_cache_set_profiling.argtypes = [vp, i32]
@@ -198,6 +200,19 @@ class FreezeCache:
 
     def poll_status(self) -> None:
         _check(self._lib.fi_cache_poll_status(self._h))
+
+    # -- fi_cache_compute_threshold
+    def compute_threshold(self, val_acts: torch.Tensor, model_labels: torch.Tensor):
+        """ComputeThresholds for this layer: (threshold now set on the cache, number of wrong look-ups)."""
+        self._check_vecs(val_acts)
+        if model_labels.dtype != torch.int32 or model_labels.device != self.device \
+                or model_labels.numel() != val_acts.shape[0]:
+            raise ValueError("model_labels must be int32 on the cache's device, one per validation item")
+        tau, wrong = ctypes.c_float(0.0), ctypes.c_int64(0)
+        _check(self._lib.fi_cache_compute_threshold(self._h, _dp(val_acts), val_acts.stride(0), _dp(model_labels),
+                                                    val_acts.shape[0], ctypes.byref(tau), ctypes.byref(wrong),
+                                                    _stream_ptr(self.device)))
+        return float(tau.value), int(wrong.value)
 
     # -- fi_cache_set_profiling / fi_cache_read_profile
     def set_profiling(self, enable: bool) -> None:

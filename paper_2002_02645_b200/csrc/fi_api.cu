@@ -59,6 +59,7 @@ void free_all(fi_cache *c) {
     cudaFree(c->slot_hit);
     cudaFree(c->plan_dev);
     cudaFree(c->row_bound);
+    cudaFree(c->calib_acc);
     cudaFree(c->status_dev);
     cudaFree(c->h2d_stage);
     if (c->copy_ev) {
@@ -584,6 +585,48 @@ fi_status_t fi_cascade_run_host(fi_cache_t *const *caches, int32_t num_stages, c
     e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return cuda_fail(e, "fi_cascade_run_host: synchronising");
     if (stage_arrivals_host) stage_arrivals_host[0] = batch0;
+    return FI_OK;
+}
+
+fi_status_t fi_cache_compute_threshold(fi_cache_t *c, const void *val_acts, int64_t ld_elems, const int32_t *model_labels,
+                                       int64_t n, float *tau_out, int64_t *wrong_out, void *cuda_stream) {
+    if (!c || n < 0 || (n > 0 && (!val_acts || !model_labels))) {
+        set_error("fi_cache_compute_threshold: null or negative argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(c->cfg.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // two accumulator words (maximum as a bit pattern, count of wrong look-ups), allocated on first use
+    if (!c->calib_acc) {
+        fi_status_t st = dev_alloc(&c->calib_acc, 2, "allocating the calibration accumulator");
+        if (st != FI_OK) return st;
+    }
+    cudaError_t e = cudaMemsetAsync(c->calib_acc, 0, 2 * sizeof(int32_t), stream);
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cache_compute_threshold: clearing the accumulator");
+    fi_lookup_out_t out;
+    out.label = c->slot_label;
+    out.conf = c->slot_conf;
+    out.hit = c->slot_hit;
+    out.topk_dist = nullptr;
+    out.topk_idx = nullptr;
+    const unsigned char *base = static_cast<const unsigned char *>(val_acts);
+    for (int64_t lo = 0; lo < n; lo += c->cfg.max_batch) {
+        const int32_t b = (int32_t)((n - lo) < c->cfg.max_batch ? (n - lo) : c->cfg.max_batch);
+        fi_status_t st = fi_cache_lookup_batch(c, base + (size_t)lo * ld_elems * c->elem_size, ld_elems, nullptr, b,
+                                               nullptr, &out, cuda_stream);
+        if (st != FI_OK) return st;
+        st = launch_wrong_max(c->slot_label, c->slot_conf, model_labels + lo, b, c->calib_acc, stream);
+        if (st != FI_OK) return st;
+    }
+    int32_t host[2] = {0, 0};
+    e = cudaMemcpyAsync(host, c->calib_acc, sizeof host, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cache_compute_threshold: reading the result");
+    float tau;
+    memcpy(&tau, &host[0], sizeof tau);
+    c->cfg.threshold = tau;
+    if (tau_out) *tau_out = tau;
+    if (wrong_out) *wrong_out = host[1];
     return FI_OK;
 }
 

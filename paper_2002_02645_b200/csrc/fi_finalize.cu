@@ -296,7 +296,29 @@ __global__ void cascade_init_kernel(int32_t batch0, int32_t num_stages, int32_t 
     }
 }
 
+// ComputeThresholds (Pseudocode 1): running maximum of the confidences of wrong look-ups.  Confidences are
+// non-negative, so their bit patterns order like the floats and atomicMax on the pattern is a float maximum.
+__global__ void wrong_max_kernel(const int32_t *__restrict__ label, const float *__restrict__ conf,
+                                 const int32_t *__restrict__ ref, int32_t n, int32_t *__restrict__ acc) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        if (label[i] != ref[i]) {
+            atomicMax(acc, __float_as_int(fmaxf(conf[i], 0.f)));
+            atomicAdd(acc + 1, 1);
+        }
+    }
+}
+
 }  // namespace
+
+fi_status_t launch_wrong_max(const int32_t *label, const float *conf, const int32_t *ref, int32_t n, int32_t *acc,
+                             cudaStream_t stream) {
+    if (n <= 0) return FI_OK;
+    int grid = (n + 255) / 256;
+    if (grid > 1024) grid = 1024;
+    wrong_max_kernel<<<grid, 256, 0, stream>>>(label, conf, ref, n, acc);
+    count_launch();
+    return check_launch("wrong_max_kernel");
+}
 
 fi_status_t launch_finalize(const fi_cache *c, const FinalizeArgs &a, cudaStream_t stream) {
     if (a.batch_max <= 0) return FI_OK;

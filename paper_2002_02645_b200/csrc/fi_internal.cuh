@@ -113,6 +113,7 @@ struct fi_cache {
                              // CTAs of a GEMM launch (order-preserving integer image of the float)
     fi::GemmPlan *plan_dev;  // written by the GEMM kernel, read by the finalize kernel
     int32_t *status_dev;     // device status word (bounded waits that ran out)
+    int32_t *calib_acc;      // [2] threshold calibration: max wrong confidence (bit pattern), wrong count
     // staging for the host-buffer entry points (allocated on first use)
     void *h2d_stage;
     size_t h2d_stage_bytes;
@@ -165,6 +166,9 @@ fi_status_t launch_finalize(const fi_cache *c, const FinalizeArgs &a, cudaStream
 
 fi_status_t launch_compact(const fi_cache *c, const fi_cascade_state_t &st, cudaStream_t stream);
 fi_status_t launch_cascade_init(const fi_cascade_state_t &st, int32_t num_stages, cudaStream_t stream);
+// acc[0] = max(acc[0], conf[i]) as an integer image, acc[1] += 1, over the slots whose label differs from ref
+fi_status_t launch_wrong_max(const int32_t *label, const float *conf, const int32_t *ref, int32_t n, int32_t *acc,
+                             cudaStream_t stream);
 
 fi_status_t ensure_tensor_maps(fi_cache *c);
 size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, int dim);

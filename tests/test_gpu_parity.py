@@ -328,3 +328,28 @@ def test_host_lookup_matches_device_lookup():
     for a, b in zip(dev, (out.label, out.conf, out.hit, out.topk_dist, out.topk_idx)):
         np.testing.assert_array_equal(a, b.numpy())
     cache.close()
+
+
+# ------------------------------------------------------------------ ComputeThresholds on the device
+
+@pytest.mark.parametrize("path,max_batch", [(fb.FI_PATH_GEMM, 64), (fb.FI_PATH_STREAM, 200)])
+def test_compute_threshold_matches_oracle(path, max_batch):
+    w = dg.single_layer(name="t", n_cache=1500, n_query=200, dim=256, num_classes=8, dtype="bf16", sigma=0.9, k=3,
+                        seed=15)
+    st = w.stages[0]
+    # stand-in for the label the model predicts per item: the item's class, for 15 % of the items another one, so
+    # that some look-ups disagree with "the model" as they do on real validation data
+    flip = np.random.default_rng(16).random(200) < 0.15
+    model = np.where(flip, (w.query_classes + 1) % 8, w.query_classes).astype(np.int32)
+    want_tau, want_wrong = fo.compute_threshold(st.queries, st.cache_vecs, st.cache_labels, model, k=3)
+    cache = make_cache(st, k=3, num_classes=8, tau=123.0, max_batch=max_batch, path=path)    # 200 items: several batches
+    tau, wrong = cache.compute_threshold(to_device(st.queries), torch.from_numpy(model).cuda())
+    assert wrong == want_wrong and 0 < wrong < 200
+    assert tau == pytest.approx(want_tau, rel=1e-5)
+    # the cache now freezes no validation item wrongly
+    first = min(200, max_batch)
+    out = cache.lookup_batch(to_device(st.queries[:first]))
+    torch.cuda.synchronize()
+    hit = out.hit.cpu().numpy() == 1
+    assert hit.any() and (out.label.cpu().numpy()[hit] == model[:first][hit]).all()
+    cache.close()

@@ -370,3 +370,27 @@ def test_table1_memory_arithmetic():
     # the four-stage cascade workload uses exactly these activation sizes
     w = dg.config2(shrink=64)
     assert [s.dim * 64 for s in w.stages] == [64 * 32 * 32, 128 * 16 * 16, 256 * 8 * 8, 512 * 4 * 4]
+
+
+# ------------------------------------------------------------------ ComputeThresholds (Pseudocode 1, Sec. 3.1 (ii))
+
+def test_compute_threshold_hand_case_and_zero_error_property():
+    # three cached points on a line, labels 0 / 1 / 1; k = 1 so conf = 1 / squared distance
+    x = np.array([[0.0], [10.0], [20.0]], dtype=np.float32)
+    lab = np.array([0, 1, 1], dtype=np.int32)
+    v = np.array([[1.0], [9.5], [4.0], [12.0]], dtype=np.float32)         # nearest: 0, 1, 0, 1
+    model = np.array([0, 0, 1, 1], dtype=np.int32)                         # items 1 and 2 are looked up wrongly
+    tau, wrong = fo.compute_threshold(v, x, lab, model, k=1)
+    assert wrong == 2 and tau == max(1.0 / 0.25, 1.0 / 16.0)               # confidences 4 and 1/16
+    assert fo.compute_threshold(v[[0, 3]], x, lab, model[[0, 3]], k=1) == (0.0, 0)   # nothing wrong: stays at 0
+    # "zero error on the validation data": with that threshold every validation hit carries the model's label,
+    # and more validation items can only raise it
+    xs, qs, labs = _small_case(seed=13, n=300, b=120, c=5)
+    rng = np.random.default_rng(14)
+    model = np.where(rng.random(120) < 0.8, fo.lookup(qs, xs, labs, k=3, tau=0.0).label, 4).astype(np.int32)
+    tau, wrong = fo.compute_threshold(qs, xs, labs, model, k=3)
+    r = fo.lookup(qs, xs, labs, k=3, tau=tau)
+    assert wrong > 0 and (r.label[r.hit == 1] == model[r.hit == 1]).all()
+    assert tau == r.conf[r.label != model].max()
+    tau_half, _ = fo.compute_threshold(qs[:60], xs, labs, model[:60], k=3)
+    assert tau_half <= tau
