@@ -459,20 +459,63 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_kmeans(args):
+    """One Lloyd iteration at the paper's scale (Sec. 2.1 / Sec. 4): 40,000 cached points per layer reduced to 1024
+    dimensions, 200 clusters; reports points/s of fi_kmeans_step (assignment look-ups + update kernel)."""
+    import torch
+    from paper_2002_02645_b200 import binding as fb
+    from paper_2002_02645_b200 import build as fbuild
+    from paper_2002_02645_b200 import datagen as dg
+    fbuild.build_library()
+    dev = torch.device("cuda", 0)
+    n, d, clusters = 40000, 1024, 200
+    w = dg.single_layer(name="kmeans_40000x1024_200", n_cache=n, n_query=clusters, dim=d, num_classes=10, dtype="bf16",
+                        sigma=0.5, k=1, seed=0)
+    st = w.stages[0]
+    pts, labs = to_dev(st.cache_vecs, dev), torch.from_numpy(st.cache_labels).to(dev)
+    cache = fb.FreezeCache(dim=d, capacity=clusters, num_classes=10, k=1, dtype=fb.FI_BF16, max_batch=8192)
+    cache.insert(to_dev(st.queries, dev), torch.zeros(clusters, dtype=torch.int32, device=dev))
+    for _ in range(max(args.warmup, 3)):
+        cache.kmeans_step(pts, labs)
+    torch.cuda.synchronize()
+    l0 = fb.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        cache.kmeans_step(pts, labs)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    peaks, src = load_peaks()
+    nbytes = 2.0 * n * d * 2          # the points are read once by the assignment and once by the update
+    print(json.dumps({"metric": "k-means Lloyd iteration, points/s", "value": n / (ms * 1e-3), "unit": "points/s",
+                      "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+                      "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": w.name, "points": n, "dim": d, "clusters": clusters,
+                                 "l2": "points (82 MB) fit in L2: figures are L2-warm"},
+                      "gpu_launches": fb.launch_count() - l0,
+                      "roofline": {"bound": "hbm", "achieved": nbytes / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                                   "unit": "GB/s", "frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                   "peak_source": f"copy bandwidth, {src}", "traffic": None}}))
+    cache.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0", "kmeans"])
     ap.add_argument("--cpu-sample", type=int, default=0,
                     help="requests per oracle timing (0: sized for 10-30 s of CPU work)")
     ap.add_argument("--batch", type=int, default=16, help="batch of the latency workload (cfg5): 1, 4 or 16")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--same-batch", action="store_true", help="every rank serves the same batch")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.workload == "kmeans":
+        run_kmeans(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

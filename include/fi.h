@@ -124,6 +124,29 @@ fi_status_t fi_cache_set_path(fi_cache_t *cache, int32_t path);
 /* Number of entries currently stored. */
 int64_t fi_cache_size(const fi_cache_t *cache);
 
+/* Forget all entries (size becomes 0; capacity and configuration stay).  Asynchronous work already queued on the
+ * cache must have been ordered before later inserts by the caller's stream. */
+fi_status_t fi_cache_clear(fi_cache_t *cache);
+
+/*
+ * One Lloyd iteration towards the k-means cache of Sec. 4, whose entries are <cluster centre, majority label,
+ * fraction of the majority label> (Sec. 2.1 clusters each block's outputs into 200 clusters and tags them this way).
+ * `centres` is a cache that holds the current centres (its k must be 1).  Assignment step: every point goes to its
+ * nearest centre under squared L2, ties to the smaller centre index (the look-up itself, in batches of max_batch).
+ * Update step: per cluster the mean of its points, rounded to the cache's dtype; the number of points; the most
+ * frequent of the points' labels (smaller label on ties) and its share.  A cluster without points keeps its
+ * centre and gets label -1, share 0.
+ *   points [n x ld_elems] device, dtype of the cache; point_labels [n] device int32 in [0, num_classes)
+ *   assign_out [n] device int32; new_centres [size x dim] device, cache dtype; counts / majority_label [size]
+ *   device int32; fraction [size] device float
+ * Feeding (new_centres, majority_label, fraction) to fi_cache_clear + fi_cache_insert (as vecs, labels, weights)
+ * gives the next iteration's centres, and after the last iteration the k-means cache itself.  At most 8,192
+ * classes.  Asynchronous.
+ */
+fi_status_t fi_kmeans_step(fi_cache_t *centres, const void *points, int64_t ld_elems, const int32_t *point_labels,
+                           int64_t n, int32_t *assign_out, void *new_centres, int32_t *counts,
+                           int32_t *majority_label, float *fraction, void *cuda_stream);
+
 /*
  * The cache look-up API of Sec. 3 for a batch: for each request the k nearest cached entries under squared
  * L2 (ties by smaller index), per label i among them S_i = m_i/k and C_i = S_i * sum_j w_j/d_j, the label

@@ -156,6 +156,40 @@ def compute_threshold(val_queries: np.ndarray, cache: np.ndarray, labels: np.nda
     return threshold, wrong
 
 
+@dataclass
+class KMeansStep:
+    assign: np.ndarray      # [n] int64 nearest-centre index of every point
+    centres: np.ndarray     # [clusters, d] float64 means (old centre where a cluster is empty)
+    counts: np.ndarray      # [clusters] int64
+    majority: np.ndarray    # [clusters] int32, -1 for an empty cluster
+    fraction: np.ndarray    # [clusters] float64 share of the majority label
+
+
+def kmeans_step(points: np.ndarray, centres: np.ndarray, point_labels: np.ndarray, num_classes: int) -> KMeansStep:
+    """One Lloyd iteration plus the tagging of Sec. 2.1 / Sec. 4: assign every point to its nearest centre (squared
+    L2, ties to the smaller index), replace each centre by the mean of its points, and record per cluster the most
+    frequent model-predicted label (smaller label on ties) with its share."""
+    from paper_2002_02645_b200.datagen import stored_to_f64
+    clusters = centres.shape[0]
+    r = lookup(points, centres, np.zeros(clusters, np.int32), k=1, tau=0.0)
+    assign = r.ni[:, 0].copy()
+    x = stored_to_f64(points)
+    new = stored_to_f64(centres).copy()
+    counts = np.zeros(clusters, np.int64)
+    majority = np.full(clusters, -1, np.int32)
+    fraction = np.zeros(clusters, np.float64)
+    for c in range(clusters):
+        members = np.nonzero(assign == c)[0]
+        counts[c] = members.shape[0]
+        if members.shape[0] == 0:
+            continue
+        new[c] = x[members].sum(axis=0) / members.shape[0]
+        hist = np.bincount(point_labels[members], minlength=num_classes)
+        majority[c] = int(np.argmax(hist))           # first maximum = smaller label on ties
+        fraction[c] = hist[majority[c]] / members.shape[0]
+    return KMeansStep(assign, new, counts, majority, fraction)
+
+
 def compact(active: np.ndarray, hit: np.ndarray) -> np.ndarray:
     """Ids of `active` whose look-up missed, order kept (Sec. 5, batch reconstruction)."""
     a = np.ascontiguousarray(active, dtype=np.int32)

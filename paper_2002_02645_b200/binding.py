@@ -23,7 +23,7 @@ FI_PATH_AUTO, FI_PATH_STREAM, FI_PATH_GEMM = 0, 1, 2
 EXPORTS = ["fi_cache_create", "fi_cache_destroy", "fi_cache_insert", "fi_cache_set_threshold", "fi_cache_set_path",
            "fi_cache_size", "fi_cache_lookup_batch", "fi_cascade_init", "fi_cascade_step", "fi_cache_lookup_batch_host",
            "fi_cascade_run_host", "fi_cache_poll_status", "fi_cache_set_profiling",
-           "fi_cache_read_profile", "fi_lookup_noalloc", "fi_cache_compute_threshold", "fi_launch_count", "fi_last_error", "fi_status_string"]
+           "fi_cache_read_profile", "fi_lookup_noalloc", "fi_cache_compute_threshold", "fi_cache_clear", "fi_kmeans_step", "fi_launch_count", "fi_last_error", "fi_status_string"]
 
 
 class fi_cache_config_t(ctypes.Structure):
@@ -76,6 +76,8 @@ def load_library(path: Optional[str] = None):
     lib.fi_cache_lookup_batch_host.argtypes = [vp, vp, i32, ctypes.POINTER(fi_lookup_out_t), vp]
     lib.fi_cascade_run_host.argtypes = [ctypes.POINTER(vp), i32, ctypes.POINTER(vp), i32, vp, vp, vp, vp, vp]
     lib.fi_cache_poll_status.argtypes = [vp]
+    lib.fi_cache_clear.argtypes = [vp]
+    lib.fi_kmeans_step.argtypes = [vp, vp, i64, vp, i64, vp, vp, vp, vp, vp, vp]
     lib.fi_cache_compute_threshold.argtypes = [vp, vp, i64, vp, i64, ctypes.POINTER(ctypes.c_float),
                                                ctypes.POINTER(i64), vp]
     lib.fi_lookup_noalloc.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, i32, ctypes.c_float, vp, i64, i32,
@@ -200,6 +202,26 @@ class FreezeCache:
 
     def poll_status(self) -> None:
         _check(self._lib.fi_cache_poll_status(self._h))
+
+    # -- fi_cache_clear
+    def clear(self) -> None:
+        _check(self._lib.fi_cache_clear(self._h))
+
+    # -- fi_kmeans_step
+    def kmeans_step(self, points: torch.Tensor, point_labels: torch.Tensor):
+        """One Lloyd iteration with this cache's entries as the current centres (k must be 1).
+        Returns (assignment [n], new centres [size, dim], counts [size], majority label [size], fraction [size])."""
+        self._check_vecs(points)
+        n, size = points.shape[0], self.size()
+        assign = torch.empty(max(n, 1), dtype=torch.int32, device=self.device)
+        centres = torch.empty(size, self.cfg.dim, dtype=_TORCH_DTYPE[self.cfg.dtype], device=self.device)
+        counts = torch.empty(size, dtype=torch.int32, device=self.device)
+        majority = torch.empty(size, dtype=torch.int32, device=self.device)
+        fraction = torch.empty(size, dtype=torch.float32, device=self.device)
+        _check(self._lib.fi_kmeans_step(self._h, _dp(points), points.stride(0), _dp(point_labels), n, _dp(assign),
+                                        _dp(centres), _dp(counts), _dp(majority), _dp(fraction),
+                                        _stream_ptr(self.device)))
+        return assign[:n], centres, counts, majority, fraction
 
     # -- fi_cache_compute_threshold
     def compute_threshold(self, val_acts: torch.Tensor, model_labels: torch.Tensor):

@@ -8,7 +8,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libficache.so")
-SOURCES = ["fi_api.cu", "fi_stream.cu", "fi_finalize.cu", "fi_gemm.cu", "fi_noalloc.cu"]
+SOURCES = ["fi_api.cu", "fi_stream.cu", "fi_finalize.cu", "fi_gemm.cu", "fi_noalloc.cu", "fi_kmeans.cu"]
 HEADERS = [os.path.join(CSRC, "fi_internal.cuh"), os.path.join(os.path.dirname(PKG), "include", "fi.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]

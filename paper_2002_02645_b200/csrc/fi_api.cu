@@ -60,6 +60,7 @@ void free_all(fi_cache *c) {
     cudaFree(c->plan_dev);
     cudaFree(c->row_bound);
     cudaFree(c->calib_acc);
+    cudaFree(c->km_dist);
     cudaFree(c->status_dev);
     cudaFree(c->h2d_stage);
     if (c->copy_ev) {
@@ -346,6 +347,52 @@ fi_status_t fi_cache_set_path(fi_cache_t *c, int32_t path) {
 }
 
 int64_t fi_cache_size(const fi_cache_t *c) { return c ? c->size : 0; }
+
+fi_status_t fi_cache_clear(fi_cache_t *c) {
+    if (!c) {
+        set_error("fi_cache_clear: null cache");
+        return FI_ERR_INVALID_ARG;
+    }
+    c->size = 0;
+    c->tmaps_ready = false;
+    return FI_OK;
+}
+
+fi_status_t fi_kmeans_step(fi_cache_t *c, const void *points, int64_t ld_elems, const int32_t *point_labels, int64_t n,
+                           int32_t *assign_out, void *new_centres, int32_t *counts, int32_t *majority_label,
+                           float *fraction, void *cuda_stream) {
+    if (!c || n < 0 || !new_centres || !counts || !majority_label || !fraction ||
+        (n > 0 && (!points || !point_labels || !assign_out))) {
+        set_error("fi_kmeans_step: null or negative argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    if (c->cfg.k != 1 || c->size <= 0) {
+        set_error("fi_kmeans_step: the centres cache must have k = 1 and hold at least one centre");
+        return FI_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(c->cfg.device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (!c->km_dist) {
+        fi_status_t st = dev_alloc(&c->km_dist, (size_t)c->cfg.max_batch, "allocating k-means scratch");
+        if (st != FI_OK) return st;
+    }
+    // assignment: the nearest-centre index is the look-up's single neighbour
+    fi_lookup_out_t out;
+    out.label = c->slot_label;
+    out.conf = c->slot_conf;
+    out.hit = c->slot_hit;
+    out.topk_dist = c->km_dist;
+    const unsigned char *base = static_cast<const unsigned char *>(points);
+    for (int64_t lo = 0; lo < n; lo += c->cfg.max_batch) {
+        const int32_t b = (int32_t)((n - lo) < c->cfg.max_batch ? (n - lo) : c->cfg.max_batch);
+        out.topk_idx = assign_out + lo;
+        fi_status_t st = fi_cache_lookup_batch(c, base + (size_t)lo * ld_elems * c->elem_size, ld_elems, nullptr, b,
+                                               nullptr, &out, cuda_stream);
+        if (st != FI_OK) return st;
+    }
+    return launch_kmeans_update(c, points, ld_elems, point_labels, assign_out, n, new_centres, counts, majority_label,
+                                fraction, stream);
+}
 
 fi_status_t fi_cache_lookup_batch(const fi_cache_t *cache, const void *queries, int64_t ld_elems, const int32_t *row_idx,
                                   int32_t batch_max, const int32_t *batch_count_dev, const fi_lookup_out_t *out,

@@ -114,6 +114,7 @@ struct fi_cache {
     fi::GemmPlan *plan_dev;  // written by the GEMM kernel, read by the finalize kernel
     int32_t *status_dev;     // device status word (bounded waits that ran out)
     int32_t *calib_acc;      // [2] threshold calibration: max wrong confidence (bit pattern), wrong count
+    float *km_dist;          // [max_batch] k-means assignment scratch: nearest distances of one batch (unused output)
     // staging for the host-buffer entry points (allocated on first use)
     void *h2d_stage;
     size_t h2d_stage_bytes;
@@ -169,6 +170,11 @@ fi_status_t launch_cascade_init(const fi_cascade_state_t &st, int32_t num_stages
 // acc[0] = max(acc[0], conf[i]) as an integer image, acc[1] += 1, over the slots whose label differs from ref
 fi_status_t launch_wrong_max(const int32_t *label, const float *conf, const int32_t *ref, int32_t n, int32_t *acc,
                              cudaStream_t stream);
+
+// k-means update step (means, counts, majority label and its share) for the centres held in `c`
+fi_status_t launch_kmeans_update(const fi_cache *c, const void *points, int64_t ld, const int32_t *point_labels,
+                                 const int32_t *assign, int64_t n, void *new_centres, int32_t *counts,
+                                 int32_t *majority, float *fraction, cudaStream_t stream);
 
 fi_status_t ensure_tensor_maps(fi_cache *c);
 size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, int dim);

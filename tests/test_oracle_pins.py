@@ -394,3 +394,44 @@ def test_compute_threshold_hand_case_and_zero_error_property():
     assert tau == r.conf[r.label != model].max()
     tau_half, _ = fo.compute_threshold(qs[:60], xs, labs, model[:60], k=3)
     assert tau_half <= tau
+
+
+# ------------------------------------------------------------------ k-means cache construction (Sec. 2.1, Sec. 4)
+
+def test_kmeans_step_hand_case_ties_and_empty_cluster():
+    pts = np.array([[0.0], [1.0], [2.0], [10.0], [11.0], [5.5]], dtype=np.float32)
+    lab = np.array([3, 3, 1, 2, 2, 1], dtype=np.int32)
+    cen = np.array([[1.0], [10.0], [100.0]], dtype=np.float32)
+    s = fo.kmeans_step(pts, cen, lab, num_classes=4)
+    # 5.5 is equally far from 1 and 10: ties go to the smaller centre index
+    assert list(s.assign) == [0, 0, 0, 1, 1, 0]
+    np.testing.assert_allclose(s.centres[:, 0], [(0 + 1 + 2 + 5.5) / 4, 10.5, 100.0])     # the empty cluster keeps its centre
+    assert list(s.counts) == [4, 2, 0]
+    # cluster 0 holds labels 3, 3, 1, 1: a tie, the smaller label wins with share 2/4
+    assert list(s.majority) == [1, 2, -1] and list(s.fraction) == [0.5, 1.0, 0.0]
+
+
+def test_kmeans_step_against_sklearn_and_invariants():
+    from sklearn.cluster import KMeans
+    rng = np.random.default_rng(21)
+    true = rng.normal(size=(6, 12)) * 4
+    lab = rng.integers(0, 6, 900).astype(np.int32)
+    pts = (true[lab] + rng.normal(size=(900, 12))).astype(np.float32)
+    init = pts[rng.choice(900, 6, replace=False)].copy()
+    s = fo.kmeans_step(pts, init, lab, num_classes=6)
+    km = KMeans(n_clusters=6, init=init.astype(np.float64), n_init=1, max_iter=1, tol=0.0, algorithm="lloyd").fit(
+        pts.astype(np.float64))
+    np.testing.assert_allclose(s.centres, km.cluster_centers_, rtol=1e-9, atol=1e-9)
+    assert s.counts.sum() == 900
+    np.testing.assert_allclose((s.centres * s.counts[:, None]).sum(0) / 900, pts.astype(np.float64).mean(0), rtol=1e-12)
+    # Lloyd iterations never increase the within-cluster sum of squares
+    cen, inertia = init, []
+    for _ in range(4):
+        st = fo.kmeans_step(pts, cen, lab, num_classes=6)
+        inertia.append(((pts.astype(np.float64) - cen.astype(np.float64)[st.assign]) ** 2).sum())
+        cen = st.centres.astype(np.float32)
+    assert all(a >= b * (1 - 1e-6) for a, b in zip(inertia, inertia[1:]))
+    # the majority share of a non-empty cluster lies in [1/classes, 1]; clusters that caught a single blob are pure
+    # (Sec. 2.1's observation on cluster purity)
+    live = st.counts > 0
+    assert (st.fraction[live] >= 1.0 / 6).all() and (st.fraction[live] <= 1.0).all() and (st.fraction[live] > 0.95).any()
