@@ -59,6 +59,7 @@ void free_all(fi_cache *c) {
     cudaFree(c->slot_hit);
     cudaFree(c->plan_dev);
     cudaFree(c->row_bound);
+    cudaFree(c->tail_dump);
     cudaFree(c->calib_acc);
     cudaFree(c->km_dist);
     cudaFree(c->status_dev);

@@ -191,25 +191,91 @@ struct TopList {
     }
 };
 
-struct TileWalk {
-    // cache-row range of this CTA and how it is cut into tiles
-    int col_begin, col_end, tiles, tile_w;
-    __device__ __forceinline__ void setup(const GemmPlan &p, int q, long long n_entries) {
-        long long n_pad = ((n_entries + 15) / 16) * 16;
-        long long b = (long long)q * p.range16 * 16;
-        long long e = b + (long long)p.range16 * 16;
-        if (e > n_pad) e = n_pad;
-        if (b > e) b = e;
-        col_begin = (int)b;
-        col_end = (int)e;
-        int cols = col_end - col_begin;
-        tiles = (cols + kMaxTileN - 1) / kMaxTileN;
-        tile_w = tiles > 0 ? (((cols + tiles - 1) / tiles + 15) / 16) * 16 : 0;
+// One unit of work of a CTA: a tile of `w` cache rows starting at `col0` against query tile `m_tile`, over the
+// k-blocks [kb0, kb1).  `select` tiles feed the per-row lists (reset before the first tile of a list, emitted
+// after the last); the others store their partial sums for the tail kernel.
+struct WorkItem {
+    int m_tile, col0, w, kb0, kb1;
+    int list;        // list index the rows' candidates go to (select tiles)
+    int dump_slot;   // slot of the partial sums (tail pieces)
+    bool select, reset, emit;
+};
+
+struct Schedule {
+    GemmPlan plan;
+    int cta, num_ctas, m_local, q, num_kb;
+    long long n16;
+    // ranges mode
+    int col_begin, col_end, tiles, tile_w, my_groups;
+
+    __device__ __forceinline__ void setup(const GemmPlan &p, int cta_, int num_ctas_, long long n_entries, int num_kb_) {
+        plan = p;
+        cta = cta_;
+        num_ctas = num_ctas_;
+        num_kb = num_kb_;
+        n16 = (n_entries + 15) / 16;
+        m_local = cta % p.mg;
+        q = cta / p.mg;
+        col_begin = col_end = tiles = tile_w = my_groups = 0;
+        if (p.mode == 0 && p.m_tiles > 0 && p.range16 > 0 && q < p.parts) {
+            long long b = (long long)q * p.range16, e = b + p.range16;
+            if (e > n16) e = n16;
+            if (b > e) b = e;
+            col_begin = (int)(b * 16);
+            col_end = (int)(e * 16);
+            const int cols = col_end - col_begin;
+            tiles = (cols + kMaxTileN - 1) / kMaxTileN;
+            tile_w = tiles > 0 ? (((cols + tiles - 1) / tiles + 15) / 16) * 16 : 0;
+            my_groups = m_local < p.m_tiles ? (p.m_tiles - m_local + p.mg - 1) / p.mg : 0;
+        }
     }
-    __device__ __forceinline__ int col0(int t) const { return col_begin + t * tile_w; }
-    __device__ __forceinline__ int width(int t) const {
-        int w = col_end - col0(t);
-        return w < tile_w ? w : tile_w;
+    // widest tile this CTA will load (sizes the shared-memory stages)
+    __device__ __forceinline__ int max_width() const { return plan.mode == 0 ? tile_w : kMaxTileN; }
+    __device__ __forceinline__ int num_items() const {
+        if (plan.m_tiles == 0 || n16 == 0) return 0;
+        if (plan.mode == 0) return my_groups * tiles;
+        return 1 + (cta < plan.tail_tiles * plan.tail_slices ? 1 : 0);
+    }
+    // wave + tail: the id-th tile in (cache-row tile, query tile) order; cache-row tiles are as even as 16-row
+    // blocks allow
+    __device__ __forceinline__ void tile_of(int id, WorkItem &it) const {
+        const int n = id / plan.m_tiles;
+        it.m_tile = id % plan.m_tiles;
+        const long long b0 = n16 * n / plan.n_tiles, b1 = n16 * (n + 1) / plan.n_tiles;
+        it.col0 = (int)(b0 * 16);
+        it.w = (int)((b1 - b0) * 16);
+        it.list = n;
+    }
+    // idx-th item; g and t are the caller's running (group, tile) counters in ranges mode (no divisions on the
+    // hand-over path between tiles)
+    __device__ __forceinline__ void item(int idx, int g, int t, WorkItem &it) const {
+        it.dump_slot = 0;
+        if (plan.mode == 0) {
+            it.m_tile = g * plan.mg + m_local;
+            it.col0 = col_begin + t * tile_w;
+            const int rest = col_end - it.col0;
+            it.w = rest < tile_w ? rest : tile_w;
+            it.kb0 = 0;
+            it.kb1 = num_kb;
+            it.list = q;
+            it.select = true;
+            it.reset = t == 0;
+            it.emit = t == tiles - 1;
+            return;
+        }
+        if (idx == 0) {
+            tile_of(cta, it);
+            it.kb0 = 0;
+            it.kb1 = num_kb;
+            it.select = it.reset = it.emit = true;
+            return;
+        }
+        const int j = cta / plan.tail_slices, sl = cta % plan.tail_slices;
+        tile_of(num_ctas + j, it);
+        it.kb0 = (int)((long long)num_kb * sl / plan.tail_slices);
+        it.kb1 = (int)((long long)num_kb * (sl + 1) / plan.tail_slices);
+        it.select = it.reset = it.emit = false;
+        it.dump_slot = cta;
     }
 };
 
@@ -220,7 +286,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                    const __grid_constant__ CUtensorMap tmap_x16, const float *__restrict__ norms, long long n_entries,
                    int dim, int batch_max, const int32_t *__restrict__ count_dev, int k,
                    float *__restrict__ part_score, int32_t *__restrict__ part_idx, GemmPlan *__restrict__ plan_out,
-                   int32_t *row_bound, int32_t *__restrict__ status) {
+                   int32_t *row_bound, float *__restrict__ tail_dump, int32_t *__restrict__ status) {
     constexpr int kTileRows = kTileM * MSUB;
     constexpr int kATileBytes = kABytes * MSUB;
     constexpr int kAccBufs = MSUB == 1 ? 2 : 1;   // accumulator sets in TMEM
@@ -235,28 +301,23 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     SmemCtl *ctl = reinterpret_cast<SmemCtl *>(smem + kStageRegionBytes + kNormSmemBytes + kQueueSmemBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_kb = (dim + kBlockK - 1) / kBlockK;
 
     if (threadIdx.x == 0) {
         int count = count_dev ? min(*count_dev, batch_max) : batch_max;
         if (count < 0) count = 0;
-        ctl->plan = make_gemm_plan(count, n_entries, (int)gridDim.x, k, kTileRows);
+        ctl->plan = make_gemm_plan(count, n_entries, (int)gridDim.x, k, kTileRows, num_kb);
         ctl->abort_flag = 0;
         if (blockIdx.x == 0) *plan_out = ctl->plan;
     }
     __syncthreads();
-    const GemmPlan plan = ctl->plan;
-    const int m_local = blockIdx.x % plan.mg;
-    const int q = blockIdx.x / plan.mg;
-    if (plan.m_tiles == 0 || plan.range16 == 0 || q >= plan.parts) return;   // whole CTA, before any barrier
-    TileWalk walk;
-    walk.setup(plan, q, n_entries);
-    if (walk.tiles == 0) return;
-    const int num_kb = (dim + kBlockK - 1) / kBlockK;
-    // groups in which this CTA has a query tile: a prefix of all groups
-    const int my_groups = m_local < plan.m_tiles ? (plan.m_tiles - m_local + plan.mg - 1) / plan.mg : 0;
-    if (my_groups == 0) return;
+    Schedule sched;
+    sched.setup(ctl->plan, (int)blockIdx.x, (int)gridDim.x, n_entries, num_kb);
+    const GemmPlan &plan = sched.plan;
+    const int n_items = sched.num_items();
+    if (n_items == 0) return;   // whole CTA, before any barrier
     // as many stages as fit: narrower tiles leave room for a deeper ring
-    const int stage_bytes = kATileBytes + walk.tile_w * (kBlockK * 2);
+    const int stage_bytes = kATileBytes + sched.max_width() * (kBlockK * 2);
     const int num_stages = min(kMaxStages, kStageRegionBytes / stage_bytes);
 
     if (threadIdx.x == 0) {
@@ -285,39 +346,49 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t it = 0, stage = 0, ph = 0;
+            uint32_t issued = 0, stage = 0, ph = 0;
             bool ok = true;
-            for (int g = 0; g < my_groups && ok; ++g) {
-                const int m_tile = g * plan.mg + m_local;
-                for (int t = 0; t < walk.tiles && ok; ++t) {
-                    const int col0 = walk.col0(t), w = walk.width(t);
-                    for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                        if (!mbar_wait(&ctl->empty[stage], ph ^ 1, ctl, status, 1)) {
-                            ok = false;
-                            break;
-                        }
-                        mbar_expect_tx(&ctl->full[stage], (uint32_t)(kATileBytes + w * kBlockK * 2));
-                        const uint32_t a_dst = smem_u32(stage_base + stage * stage_bytes);
-                        const uint32_t b_dst = a_dst + kATileBytes;
-#pragma unroll
-                        for (int ms = 0; ms < MSUB; ++ms)
-                            tma_load_2d(a_dst + ms * kABytes, &tmap_q, &ctl->full[stage], kb * kBlockK,
-                                        m_tile * kTileRows + ms * kTileM);
-                        int r = 0;
-                        for (; r + 64 <= w; r += 64)
-                            tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x64, &ctl->full[stage], kb * kBlockK, col0 + r);
-                        for (; r < w; r += 16)
-                            tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x16, &ctl->full[stage], kb * kBlockK, col0 + r);
-                        if (++stage == (uint32_t)num_stages) {
-                            stage = 0;
-                            ph ^= 1;
-                        }
+            // all k-blocks [kb0, kb1) of one tile
+            auto load_tile = [&](int m_tile, int col0, int w, int kb0, int kb1) {
+                for (int kb = kb0; kb < kb1; ++kb, ++issued) {
+                    if (!mbar_wait(&ctl->empty[stage], ph ^ 1, ctl, status, 1)) {
+                        ok = false;
+                        break;
                     }
+                    mbar_expect_tx(&ctl->full[stage], (uint32_t)(kATileBytes + w * kBlockK * 2));
+                    const uint32_t a_dst = smem_u32(stage_base + stage * stage_bytes);
+                    const uint32_t b_dst = a_dst + kATileBytes;
+#pragma unroll
+                    for (int ms = 0; ms < MSUB; ++ms)
+                        tma_load_2d(a_dst + ms * kABytes, &tmap_q, &ctl->full[stage], kb * kBlockK,
+                                    m_tile * kTileRows + ms * kTileM);
+                    int r = 0;
+                    for (; r + 64 <= w; r += 64)
+                        tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x64, &ctl->full[stage], kb * kBlockK, col0 + r);
+                    for (; r < w; r += 16)
+                        tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x16, &ctl->full[stage], kb * kBlockK, col0 + r);
+                    if (++stage == (uint32_t)num_stages) {
+                        stage = 0;
+                        ph ^= 1;
+                    }
+                }
+            };
+            if (plan.mode == 0) {
+                for (int g = 0; g < sched.my_groups && ok; ++g)
+                    for (int t = 0; t < sched.tiles && ok; ++t) {
+                        const int col0 = sched.col_begin + t * sched.tile_w;
+                        load_tile(g * plan.mg + sched.m_local, col0, min(sched.tile_w, sched.col_end - col0), 0, num_kb);
+                    }
+            } else {
+                for (int idx = 0; idx < n_items && ok; ++idx) {
+                    WorkItem it;
+                    sched.item(idx, 0, 0, it);
+                    load_tile(it.m_tile, it.col0, it.w, it.kb0, it.kb1);
                 }
             }
             if (!ok) {
                 // gave up: let the copies already issued land before the CTA leaves
-                uint32_t back = it < (uint32_t)num_stages ? it : (uint32_t)num_stages;
+                uint32_t back = issued < (uint32_t)num_stages ? issued : (uint32_t)num_stages;
                 uint32_t s2 = stage, p2 = ph;
                 for (uint32_t j = 0; j < back; ++j) {
                     if (s2 == 0) {
@@ -334,41 +405,51 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            uint32_t tile_no = 0, stage = 0, ph = 0;
+            uint32_t stage = 0, ph = 0, tile_no = 0;
             bool ok = true;
-            for (int g = 0; g < my_groups && ok; ++g) {
-                for (int t = 0; t < walk.tiles && ok; ++t, ++tile_no) {
-                    const int w = walk.width(t);
-                    const uint32_t acc = tile_no % kAccBufs, acc_ph = (tile_no / kAccBufs) & 1;
-                    if (!mbar_wait(&ctl->tmem_empty[acc], acc_ph ^ 1, ctl, status, 2)) {
+            // all MMAs of one tile over the k-blocks [kb0, kb1)
+            auto mma_tile = [&](int w, int kb0, int kb1) {
+                const uint32_t acc = tile_no % kAccBufs, acc_ph = (tile_no / kAccBufs) & 1;
+                ++tile_no;
+                if (!mbar_wait(&ctl->tmem_empty[acc], acc_ph ^ 1, ctl, status, 2)) {
+                    ok = false;
+                    return;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * kMaxTileN;
+                const uint32_t idesc = umma_instr_desc(w);
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    if (!mbar_wait(&ctl->full[stage], ph, ctl, status, 3)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + acc * kMaxTileN;
-                    const uint32_t idesc = umma_instr_desc(w);
-                    for (int kb = 0; kb < num_kb; ++kb) {
-                        if (!mbar_wait(&ctl->full[stage], ph, ctl, status, 3)) {
-                            ok = false;
-                            break;
-                        }
-                        tc_fence_after();
-                        const uint32_t a_addr = smem_u32(stage_base + stage * stage_bytes);
-                        const uint64_t bdesc = umma_smem_desc(a_addr + kATileBytes);
+                    const uint32_t a_addr = smem_u32(stage_base + stage * stage_bytes);
+                    const uint64_t bdesc = umma_smem_desc(a_addr + kATileBytes);
 #pragma unroll
-                        for (int kk = 0; kk < kBlockK / 16; ++kk) {
+                    for (int kk = 0; kk < kBlockK / 16; ++kk) {
 #pragma unroll
-                            for (int ms = 0; ms < MSUB; ++ms)
-                                umma_bf16(d_tmem + ms * kMaxTileN, umma_smem_desc(a_addr + ms * kABytes) + 2 * kk,
-                                          bdesc + 2 * kk, idesc, (kb | kk) != 0);
-                        }
-                        umma_commit(&ctl->empty[stage]);   // frees the stage once these MMAs have read it
-                        if (++stage == (uint32_t)num_stages) {
-                            stage = 0;
-                            ph ^= 1;
-                        }
+                        for (int ms = 0; ms < MSUB; ++ms)
+                            umma_bf16(d_tmem + ms * kMaxTileN, umma_smem_desc(a_addr + ms * kABytes) + 2 * kk,
+                                      bdesc + 2 * kk, idesc, ((kb - kb0) | kk) != 0);
                     }
-                    if (ok) umma_commit(&ctl->tmem_full[acc]);
+                    umma_commit(&ctl->empty[stage]);   // frees the stage once these MMAs have read it
+                    if (++stage == (uint32_t)num_stages) {
+                        stage = 0;
+                        ph ^= 1;
+                    }
+                }
+                if (ok) umma_commit(&ctl->tmem_full[acc]);
+            };
+            if (plan.mode == 0) {
+                for (int g = 0; g < sched.my_groups && ok; ++g)
+                    for (int t = 0; t < sched.tiles && ok; ++t)
+                        mma_tile(min(sched.tile_w, sched.col_end - (sched.col_begin + t * sched.tile_w)), 0, num_kb);
+            } else {
+                for (int idx = 0; idx < n_items && ok; ++idx) {
+                    WorkItem it;
+                    sched.item(idx, 0, 0, it);
+                    mma_tile(it.w, it.kb0, it.kb1);
                 }
             }
         }
@@ -386,7 +467,6 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         float *qs = queue_s + te;
         int32_t *qi = queue_i + te;
         TopList<KP> top;
-        uint32_t tile_no = 0;
         bool ok = true;
 
         // Bound shared by every CTA that scans cache rows for the same query: each list publishes its list_len-th
@@ -406,113 +486,154 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             }
         };
 
-        for (int g = 0; g < my_groups && ok; ++g) {
-            const int m_tile = g * plan.mg + m_local;
-            int32_t *my_bound = row_bound + m_tile * kTileRows + row_in_tile;
-            top.reset();
-            for (int t = 0; t < walk.tiles && ok; ++t, ++tile_no) {
-                const int col0 = walk.col0(t), w = walk.width(t);
-                const uint32_t acc = tile_no % kAccBufs, acc_ph = (tile_no / kAccBufs) & 1;
-                float *nrm = my_norm + acc * (kMaxTileN / 2);   // acc is 0 for 256-row tiles
-                int32_t bound_key;   // read past L1: other SMs lower it
-                asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(bound_key) : "l"(my_bound) : "memory");
-                // squared norms of this warp's columns, chunk after chunk; rows past the end of the cache get +inf
-                // and never enter a list
-                for (int li = lane;; li += 32) {
-                    const int c = first + (li >> 4) * kStep + (li & 15);
-                    if (c - (li & 15) >= w) break;
-                    nrm[li] = (long long)(col0 + c) < n_entries ? __ldg(norms + col0 + c) : __int_as_float(0x7F800000);
-                }
-                __syncwarp();
-                // the whole warp takes the same decision, so its lanes stay together for the TMEM loads
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, status, 4));
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (acc + msub) * kMaxTileN;
-                bound = key_float(bound_key);
-                float thr = fminf(top.s[KP - 1], bound);   // pre-filter: nothing above it can enter the list
-                int cnt = 0;
+        uint32_t tile_no = 0;
 
-                auto process = [&](const uint32_t (&v)[16], int c0, int li0) {
-                    const float4 *n4 = reinterpret_cast<const float4 *>(nrm + li0);
-                    const float4 na = n4[0], nb = n4[1], nc = n4[2], nd = n4[3];
-                    const float nv[16] = {na.x, na.y, na.z, na.w, nb.x, nb.y, nb.z, nb.w,
-                                          nc.x, nc.y, nc.z, nc.w, nd.x, nd.y, nd.z, nd.w};
-                    float sc[16];
+        // scan one accumulator tile into the running list of this thread's row
+        auto select_tile = [&](int m_tile, int col0, int w) {
+            const uint32_t acc = tile_no % kAccBufs, acc_ph = (tile_no / kAccBufs) & 1;
+            ++tile_no;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (acc + msub) * kMaxTileN;
+            int32_t *my_bound = row_bound + m_tile * kTileRows + row_in_tile;
+            float *nrm = my_norm + acc * (kMaxTileN / 2);   // acc is 0 for 256-row tiles
+            int32_t bound_key;   // read past L1: other SMs lower it
+            asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(bound_key) : "l"(my_bound) : "memory");
+            // squared norms of this warp's columns, chunk after chunk; rows past the end of the cache get +inf
+            // and never enter a list
+            for (int li = lane;; li += 32) {
+                const int c = first + (li >> 4) * kStep + (li & 15);
+                if (c - (li & 15) >= w) break;
+                nrm[li] = (long long)(col0 + c) < n_entries ? __ldg(norms + col0 + c) : __int_as_float(0x7F800000);
+            }
+            __syncwarp();
+            // the whole warp takes the same decision, so its lanes stay together for the TMEM loads
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, status, 4));
+            if (!ok) return;
+            tc_fence_after();
+            bound = key_float(bound_key);
+            float thr = fminf(top.s[KP - 1], bound);   // pre-filter: nothing above it can enter the list
+            int cnt = 0;
+
+            auto process = [&](const uint32_t (&v)[16], int c0, int li0) {
+                const float4 *n4 = reinterpret_cast<const float4 *>(nrm + li0);
+                const float4 na = n4[0], nb = n4[1], nc = n4[2], nd = n4[3];
+                const float nv[16] = {na.x, na.y, na.z, na.w, nb.x, nb.y, nb.z, nb.w,
+                                      nc.x, nc.y, nc.z, nc.w, nd.x, nd.y, nd.z, nd.w};
+                float sc[16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) sc[j] = fmaf(-2.f, __uint_as_float(v[j]), nv[j]);
-                    float m0 = fminf(fminf(sc[0], sc[1]), fminf(sc[2], sc[3]));
-                    float m1 = fminf(fminf(sc[4], sc[5]), fminf(sc[6], sc[7]));
-                    float m2 = fminf(fminf(sc[8], sc[9]), fminf(sc[10], sc[11]));
-                    float m3 = fminf(fminf(sc[12], sc[13]), fminf(sc[14], sc[15]));
-                    const float mn = fminf(fminf(m0, m1), fminf(m2, m3));
-                    const int cnt0 = cnt;
-                    if (mn <= thr) {
+                for (int j = 0; j < 16; ++j) sc[j] = fmaf(-2.f, __uint_as_float(v[j]), nv[j]);
+                float m0 = fminf(fminf(sc[0], sc[1]), fminf(sc[2], sc[3]));
+                float m1 = fminf(fminf(sc[4], sc[5]), fminf(sc[6], sc[7]));
+                float m2 = fminf(fminf(sc[8], sc[9]), fminf(sc[10], sc[11]));
+                float m3 = fminf(fminf(sc[12], sc[13]), fminf(sc[14], sc[15]));
+                const float mn = fminf(fminf(m0, m1), fminf(m2, m3));
+                const int cnt0 = cnt;
+                if (mn <= thr) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            if (sc[j] <= thr) {
-                                if (cnt < kQueueCap) {
-                                    qs[cnt * kEpiThreads] = sc[j];
-                                    qi[cnt * kEpiThreads] = col0 + c0 + j;
-                                }
-                                ++cnt;
+                    for (int j = 0; j < 16; ++j) {
+                        if (sc[j] <= thr) {
+                            if (cnt < kQueueCap) {
+                                qs[cnt * kEpiThreads] = sc[j];
+                                qi[cnt * kEpiThreads] = col0 + c0 + j;
                             }
+                            ++cnt;
                         }
                     }
-                    if (__any_sync(0xFFFFFFFFu, cnt > kQueueCap)) {
-                        // a queue overflowed inside this chunk: insert what was queued before it, then this chunk
-                        // column by column (arrival order, hence the tie order, is kept)
-                        flush(cnt0);
+                }
+                if (__any_sync(0xFFFFFFFFu, cnt > kQueueCap)) {
+                    // a queue overflowed inside this chunk: insert what was queued before it, then this chunk
+                    // column by column (arrival order, hence the tie order, is kept)
+                    flush(cnt0);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (sc[j] < top.s[KP - 1] && sc[j] <= bound) top.insert(sc[j], col0 + c0 + j);
-                        cnt = 0;
-                        thr = fminf(top.s[KP - 1], bound);
-                    }
-                };
+                    for (int j = 0; j < 16; ++j)
+                        if (sc[j] < top.s[KP - 1] && sc[j] <= bound) top.insert(sc[j], col0 + c0 + j);
+                    cnt = 0;
+                    thr = fminf(top.s[KP - 1], bound);
+                }
+            };
 
-                // two register buffers: the TMEM load of the next chunk is in flight while this one is scanned
-                uint32_t va[16], vb[16];
-                int c0 = first, li0 = 0;
-                if (c0 < w) {
-                    __syncwarp();
-                    tmem_ld16(taddr + c0, va);
-                }
-                while (c0 < w) {
-                    tmem_ld_wait(va);
-                    if (c0 + kStep < w) {
-                        __syncwarp();
-                        tmem_ld16(taddr + c0 + kStep, vb);
-                    }
-                    process(va, c0, li0);
-                    c0 += kStep;
-                    li0 += 16;
-                    if (c0 >= w) break;
-                    tmem_ld_wait(vb);
-                    if (c0 + kStep < w) {
-                        __syncwarp();
-                        tmem_ld16(taddr + c0 + kStep, va);
-                    }
-                    process(vb, c0, li0);
-                    c0 += kStep;
-                    li0 += 16;
-                }
-                tc_fence_before();
-                mbar_arrive(&ctl->tmem_empty[acc]);
-                flush(cnt);   // after the accumulator is released: the MMAs of the next tile can start meanwhile
-                if (top.s[KP - 1] < bound) atomicMin(my_bound, float_key(top.s[KP - 1]));
+            // two register buffers: the TMEM load of the next chunk is in flight while this one is scanned
+            uint32_t va[16], vb[16];
+            int c0 = first, li0 = 0;
+            if (c0 < w) {
                 __syncwarp();
+                tmem_ld16(taddr + c0, va);
             }
-            if (ok) {
-                const int row = m_tile * kTileRows + row_in_tile;
-                if (row < plan.count) {
-                    const int list = MSUB == 1 ? q * 2 + half : q;
-                    const long long o = ((long long)row * plan.lists + list) * KP;
+            while (c0 < w) {
+                tmem_ld_wait(va);
+                if (c0 + kStep < w) {
+                    __syncwarp();
+                    tmem_ld16(taddr + c0 + kStep, vb);
+                }
+                process(va, c0, li0);
+                c0 += kStep;
+                li0 += 16;
+                if (c0 >= w) break;
+                tmem_ld_wait(vb);
+                if (c0 + kStep < w) {
+                    __syncwarp();
+                    tmem_ld16(taddr + c0 + kStep, va);
+                }
+                process(vb, c0, li0);
+                c0 += kStep;
+                li0 += 16;
+            }
+            tc_fence_before();
+            mbar_arrive(&ctl->tmem_empty[acc]);
+            flush(cnt);   // after the accumulator is released: the MMAs of the next tile can start meanwhile
+            if (top.s[KP - 1] < bound) atomicMin(my_bound, float_key(top.s[KP - 1]));
+            __syncwarp();
+        };
+
+        // write this thread's list as list number `list` of its row
+        auto emit_list = [&](int m_tile, int list) {
+            const int row = m_tile * kTileRows + row_in_tile;
+            if (row < plan.count) {
+                const long long o = ((long long)row * plan.lists + list) * KP;
 #pragma unroll
-                    for (int e = 0; e < KP; ++e) {
-                        part_score[o + e] = top.s[e];
-                        part_idx[o + e] = top.i[e];
+                for (int e = 0; e < KP; ++e) {
+                    part_score[o + e] = top.s[e];
+                    part_idx[o + e] = top.i[e];
+                }
+            }
+        };
+
+        if (plan.mode == 0) {
+            for (int g = 0; g < sched.my_groups && ok; ++g) {
+                const int m_tile = g * plan.mg + sched.m_local;
+                top.reset();
+                for (int t = 0; t < sched.tiles && ok; ++t) {
+                    const int col0 = sched.col_begin + t * sched.tile_w;
+                    select_tile(m_tile, col0, min(sched.tile_w, sched.col_end - col0));
+                }
+                if (ok) emit_list(m_tile, MSUB == 1 ? sched.q * 2 + half : sched.q);
+            }
+        } else {
+            WorkItem it;
+            sched.item(0, 0, 0, it);
+            top.reset();
+            select_tile(it.m_tile, it.col0, it.w);
+            if (ok) emit_list(it.m_tile, it.list);
+            if (ok && n_items > 1) {
+                // tail piece: store the partial sums, column-major so that the 32 rows of a warp coalesce
+                sched.item(1, 0, 0, it);
+                const uint32_t acc = tile_no % kAccBufs, acc_ph = (tile_no / kAccBufs) & 1;
+                ++tile_no;
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (acc + msub) * kMaxTileN;
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, status, 5));
+                if (ok) {
+                    tc_fence_after();
+                    float *dst = tail_dump + ((long long)it.dump_slot * kMaxTileN) * kTileRows + row_in_tile;
+                    for (int c0 = first; c0 < it.w; c0 += kStep) {
+                        uint32_t v[16];
+                        __syncwarp();
+                        tmem_ld16(taddr + c0, v);
+                        tmem_ld_wait(v);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) dst[(long long)(c0 + j) * kTileRows] = __uint_as_float(v[j]);
                     }
+                    tc_fence_before();
+                    mbar_arrive(&ctl->tmem_empty[acc]);
+                    __syncwarp();
                 }
             }
         }
@@ -523,6 +644,74 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// Wave + tail mode, step 1: add up the pieces of every tail tile and turn the dot products into scores, in place
+// in the first piece's slot.  Grid (tail tiles, 16 column groups), one query row per thread; the partial sums are
+// column-major, so a warp reads 128 contiguous bytes.  Pieces are added in their order: the sum does not depend on
+// timing.
+__global__ void __launch_bounds__(2 * kTileM)
+tail_reduce_kernel(const GemmPlan *__restrict__ plan_dev, int num_ctas, float *__restrict__ tail_dump,
+                   const float *__restrict__ norms, long long n_entries) {
+    const GemmPlan plan = *plan_dev;
+    if (plan.mode != 1 || (int)blockIdx.x >= plan.tail_tiles) return;
+    constexpr int kRows = 2 * kTileM;
+    const long long n16 = (n_entries + 15) / 16;
+    const int n = (num_ctas + (int)blockIdx.x) / plan.m_tiles;
+    const long long b0 = n16 * n / plan.n_tiles, b1 = n16 * (n + 1) / plan.n_tiles;
+    const int col0 = (int)(b0 * 16), w = (int)((b1 - b0) * 16);
+    const int c0 = blockIdx.y * 16;
+    if (c0 >= w) return;
+    float *base = tail_dump + ((long long)blockIdx.x * plan.tail_slices * kMaxTileN + c0) * kRows + threadIdx.x;
+    float dot[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) dot[j] = 0.f;
+    for (int sl = 0; sl < plan.tail_slices; ++sl) {
+        const float *p = base + (long long)sl * kMaxTileN * kRows;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) dot[j] += p[j * kRows];
+    }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const int c = col0 + c0 + j;
+        const float nrm = (long long)c < n_entries ? __ldg(norms + c) : __int_as_float(0x7F800000);
+        base[j * kRows] = fmaf(-2.f, dot[j], nrm);
+    }
+}
+
+// Step 2: per-row select over the scores of a tail tile.  One CTA per tail tile, one query row per thread.
+template <int KP>
+__global__ void __launch_bounds__(2 * kTileM)
+tail_select_kernel(const GemmPlan *__restrict__ plan_dev, int num_ctas, const float *__restrict__ tail_dump,
+                   long long n_entries, float *__restrict__ part_score, int32_t *__restrict__ part_idx) {
+    const GemmPlan plan = *plan_dev;
+    if (plan.mode != 1 || (int)blockIdx.x >= plan.tail_tiles) return;
+    constexpr int kRows = 2 * kTileM;
+    const long long n16 = (n_entries + 15) / 16;
+    const int id = num_ctas + blockIdx.x;
+    const int n = id / plan.m_tiles, m_tile = id % plan.m_tiles;
+    const long long b0 = n16 * n / plan.n_tiles, b1 = n16 * (n + 1) / plan.n_tiles;
+    const int col0 = (int)(b0 * 16), w = (int)((b1 - b0) * 16);
+    const int row = m_tile * kRows + threadIdx.x;
+    TopList<KP> top;
+    top.reset();
+    const float *base = tail_dump + ((long long)blockIdx.x * plan.tail_slices * kMaxTileN) * kRows + threadIdx.x;
+    for (int c0 = 0; c0 < w; c0 += 16) {
+        float sc[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) sc[j] = base[(long long)(c0 + j) * kRows];
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+            if (sc[j] < top.s[KP - 1]) top.insert(sc[j], col0 + c0 + j);
+    }
+    if (row < plan.count) {
+        const long long o = ((long long)row * plan.lists + n) * KP;
+#pragma unroll
+        for (int e = 0; e < KP; ++e) {
+            part_score[o + e] = top.s[e];
+            part_idx[o + e] = top.i[e];
+        }
     }
 }
 
@@ -565,7 +754,8 @@ fi_status_t encode_bf16_map(CUtensorMap *map, const void *base, uint64_t rows, u
 }
 
 template <int KP, int MSUB>
-fi_status_t launch_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, const int32_t *count_dev, cudaStream_t stream) {
+fi_status_t launch_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, const int32_t *count_dev, bool tail_possible,
+                      cudaStream_t stream) {
     static bool attr_set = false;
     auto kern = gemm_select_kernel<KP, MSUB>;
     if (!attr_set) {
@@ -583,20 +773,32 @@ fi_status_t launch_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, con
         return FI_ERR_CUDA;
     }
     kern<<<c->sm_count, kGemmThreads, kGemmSmemBytes, stream>>>(tq, c->tmap_rows64, c->tmap_rows16, c->norms,
-                                                                  (long long)c->size, c->cfg.dim, batch_max, count_dev,
-                                                                  c->cfg.k, c->part_score, c->part_idx, c->plan_dev,
-                                                                  c->row_bound, c->status_dev);
+                                                               (long long)c->size, c->cfg.dim, batch_max, count_dev,
+                                                               c->cfg.k, c->part_score, c->part_idx, c->plan_dev,
+                                                               c->row_bound, c->tail_dump, c->status_dev);
     count_launch();
-    return check_launch("gemm_select_kernel");
+    fi_status_t st = check_launch("gemm_select_kernel");
+    if (st != FI_OK || !tail_possible) return st;
+    // the tail kernel reads the plan the GEMM wrote and returns at once when that plan has no tail
+    tail_reduce_kernel<<<dim3(c->sm_count / 2, kMaxTileN / 16), 2 * kTileM, 0, stream>>>(c->plan_dev, c->sm_count, c->tail_dump,
+                                                                                      c->norms, (long long)c->size);
+    count_launch();
+    st = check_launch("tail_reduce_kernel");
+    if (st != FI_OK) return st;
+    tail_select_kernel<KP><<<c->sm_count / 2, 2 * kTileM, 0, stream>>>(c->plan_dev, c->sm_count, c->tail_dump,
+                                                                       (long long)c->size, c->part_score, c->part_idx);
+    count_launch();
+    return check_launch("tail_select_kernel");
 }
 
 template <int MSUB>
-fi_status_t launch_msub(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, const int32_t *count_dev, cudaStream_t stream) {
+fi_status_t launch_msub(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, const int32_t *count_dev, bool tail_possible,
+                        cudaStream_t stream) {
     switch (gemm_list_len(c->cfg.k)) {
-        case 4: return launch_kp<4, MSUB>(c, tq, batch_max, count_dev, stream);
-        case 8: return launch_kp<8, MSUB>(c, tq, batch_max, count_dev, stream);
-        case 16: return launch_kp<16, MSUB>(c, tq, batch_max, count_dev, stream);
-        default: return launch_kp<32, MSUB>(c, tq, batch_max, count_dev, stream);
+        case 4: return launch_kp<4, MSUB>(c, tq, batch_max, count_dev, tail_possible, stream);
+        case 8: return launch_kp<8, MSUB>(c, tq, batch_max, count_dev, tail_possible, stream);
+        case 16: return launch_kp<16, MSUB>(c, tq, batch_max, count_dev, tail_possible, stream);
+        default: return launch_kp<32, MSUB>(c, tq, batch_max, count_dev, tail_possible, stream);
     }
 }
 
@@ -619,13 +821,24 @@ fi_status_t ensure_tensor_maps(fi_cache *c) {
 size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, int dim) {
     size_t worst = 0;
     const int tile_m = gemm_tile_m(max_batch, dim);
+    const int num_kb = (dim + kBlockK - 1) / kBlockK;
     int m_tiles_max = (max_batch + tile_m - 1) / tile_m;
     for (int mt = 1; mt <= m_tiles_max; ++mt) {
-        GemmPlan p = make_gemm_plan(mt * tile_m, capacity, sm_count, k, tile_m);
+        GemmPlan p = make_gemm_plan(mt * tile_m, capacity, sm_count, k, tile_m, num_kb);
         size_t e = (size_t)mt * tile_m * (size_t)p.lists * (size_t)p.list_len;
         if (e > worst) worst = e;
     }
     return worst;
+}
+
+// Can a batch of at most batch_max requests against the current cache end up in wave + tail mode?
+static bool tail_mode_possible(const fi_cache *c, int batch_max) {
+    const int tile_m = gemm_tile_m(batch_max, c->cfg.dim);
+    const int num_kb = (c->cfg.dim + kBlockK - 1) / kBlockK;
+    const int m_tiles_max = (batch_max + tile_m - 1) / tile_m;
+    for (int mt = 1; mt <= m_tiles_max; ++mt)
+        if (make_gemm_plan(mt * tile_m, c->size, c->sm_count, c->cfg.k, tile_m, num_kb).mode == 1) return true;
+    return false;
 }
 
 fi_status_t launch_gemm_select(fi_cache *c, const void *queries_compact, int64_t ld_elems, int32_t batch_max,
@@ -644,8 +857,25 @@ fi_status_t launch_gemm_select(fi_cache *c, const void *queries_compact, int64_t
     CUtensorMap tq;
     st = encode_bf16_map(&tq, queries_compact, (uint64_t)batch_max, (uint64_t)c->cfg.dim, (uint64_t)ld_elems, kTileM);
     if (st != FI_OK) return st;
-    if (gemm_tile_m(batch_max, c->cfg.dim) == kTileM) return launch_msub<1>(c, tq, batch_max, count_dev, stream);
-    return launch_msub<2>(c, tq, batch_max, count_dev, stream);
+    const bool tail_possible = tail_mode_possible(c, batch_max);
+    if (tail_possible && c->tail_dump_units < (size_t)c->sm_count) {
+        // one slot of 256 x 256 partial sums per CTA; allocated the first time a shape can need it
+        cudaError_t e = cudaStreamSynchronize(stream);
+        if (e == cudaSuccess) {
+            cudaFree(c->tail_dump);
+            c->tail_dump = nullptr;
+            c->tail_dump_units = 0;
+            e = cudaMalloc(reinterpret_cast<void **>(&c->tail_dump), (size_t)c->sm_count * kMaxTileN * 2 * kTileM * sizeof(float));
+        }
+        if (e != cudaSuccess) {
+            set_error("cannot allocate the partial-sum buffer of the distance GEMM: %s", cudaGetErrorString(e));
+            cudaGetLastError();
+            return e == cudaErrorMemoryAllocation ? FI_ERR_OOM : FI_ERR_CUDA;
+        }
+        c->tail_dump_units = (size_t)c->sm_count;
+    }
+    if (gemm_tile_m(batch_max, c->cfg.dim) == kTileM) return launch_msub<1>(c, tq, batch_max, count_dev, false, stream);
+    return launch_msub<2>(c, tq, batch_max, count_dev, tail_possible, stream);
 }
 
 }  // namespace fi

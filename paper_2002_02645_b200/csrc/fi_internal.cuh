@@ -25,21 +25,32 @@ __host__ __device__ inline int gemm_list_len(int k) {
 // How the tiles of the distance GEMM are spread over the CTAs.  Query tiles (`tile_m` = 128 or 256 rows each) are
 // taken in groups of `mg`; inside a group, CTA (m_local, q) owns query tile m_local and the q-th of `parts` equal
 // ranges of cache rows, so CTAs with the same q stream the same cache rows at the same time (they meet in
-// L2) and each query row ends up with `parts` candidate lists.
+// L2) and each query row ends up with one candidate list per range ("ranges" mode).
+//
+// When the whole problem is only a little more than one 256 x 256 tile per CTA (deep rows, few queries), cutting
+// ranges would leave every CTA with two narrow tiles and the query tile read twice.  The "wave + tail" mode
+// then gives each CTA one full tile over the whole row length, and the tiles left over are cut along the row
+// length into `tail_slices` pieces, one per CTA; their partial sums go to memory and a small kernel adds them
+// up and selects.
 struct GemmPlan {
-    int32_t count;      // actual batch
-    int32_t m_tiles;    // ceil(count / tile_m)
-    int32_t mg;         // query tiles per group
-    int32_t groups;     // ceil(m_tiles / mg)
-    int32_t parts;      // cache-row ranges per query tile = candidate lists per query
-    int32_t range16;    // rows per range, in units of 16 (the last range may be shorter)
-    int32_t list_len;   // entries per candidate list
-    int32_t tile_m;     // query rows per CTA tile
-    int32_t lists;      // candidate lists per query = parts x (column halves handled by separate warps)
+    int32_t count;        // actual batch
+    int32_t m_tiles;      // ceil(count / tile_m)
+    int32_t mg;           // query tiles per group
+    int32_t groups;       // ceil(m_tiles / mg)
+    int32_t parts;        // cache-row ranges per query tile
+    int32_t range16;      // rows per range, in units of 16 (the last range may be shorter)
+    int32_t list_len;     // entries per candidate list
+    int32_t tile_m;       // query rows per CTA tile
+    int32_t lists;        // candidate lists per query
+    int32_t mode;         // 0 = ranges, 1 = wave + tail
+    int32_t n_tiles;      // wave + tail: cache-row tiles per query tile
+    int32_t tail_tiles;   // wave + tail: tiles beyond the first wave
+    int32_t tail_slices;  // wave + tail: pieces each of those is cut into along the row length
     int32_t pad;
 };
 
-__host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entries, int num_ctas, int k, int tile_m) {
+__host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entries, int num_ctas, int k, int tile_m,
+                                                   int num_kb) {
     GemmPlan p;
     p.count = count;
     p.m_tiles = (count + tile_m - 1) / tile_m;
@@ -47,12 +58,32 @@ __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entrie
     p.tile_m = tile_m;
     p.pad = 0;
     p.lists = 0;
+    p.mode = 0;
+    p.n_tiles = p.tail_tiles = p.tail_slices = 0;
     long long n16 = (n_entries + 15) / 16;
     if (p.m_tiles <= 0 || n16 <= 0) {
         p.mg = p.groups = p.parts = 1;
         p.range16 = 0;
         p.lists = tile_m == kTileM ? 2 : 1;
         return p;
+    }
+    if (tile_m == 2 * kTileM && num_kb >= 64) {
+        const long long nt = (n16 + 15) / 16;                 // tiles of at most 256 rows
+        const long long total = (long long)p.m_tiles * nt;
+        if (total > num_ctas && total <= num_ctas + num_ctas / 2) {
+            p.mode = 1;
+            p.n_tiles = (int32_t)nt;
+            p.tail_tiles = (int32_t)(total - num_ctas);
+            int slices = num_ctas / p.tail_tiles;
+            if (slices > num_kb) slices = num_kb;
+            p.tail_slices = slices;
+            p.mg = p.m_tiles;
+            p.groups = 1;
+            p.parts = (int32_t)nt;
+            p.range16 = 16;
+            p.lists = (int32_t)nt;
+            return p;
+        }
     }
     // pick the group size that needs the fewest MMA columns per CTA in total
     int best_mg = 1;
@@ -109,6 +140,8 @@ struct fi_cache {
     int32_t *slot_label;     // [max_batch] per-slot results of a cascade step
     float *slot_conf;
     uint8_t *slot_hit;
+    float *tail_dump;        // partial sums of the tail tiles: [units][256 columns][256 rows], allocated on first need
+    size_t tail_dump_units;
     int32_t *row_bound;      // [max_batch + 256] per-query upper bound of the list_len-th best score, shared by all
                              // CTAs of a GEMM launch (order-preserving integer image of the float)
     fi::GemmPlan *plan_dev;  // written by the GEMM kernel, read by the finalize kernel

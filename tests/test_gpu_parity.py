@@ -99,6 +99,7 @@ def test_stream_path_large_dim_reads_queries_in_place():
     (16, 8, 17, 5),            # a single 16-row block
     (3000, 4096, 64, 13),      # list length 16, deep K
     (2500, 136, 2200, 29),     # 18 query tiles (two groups), list length 32
+    (9990, 4096, 900, 5),      # 4 x 40 tiles of 256 x 256 on 148 SMs: one full tile per CTA plus a tail cut along K
 ])
 def test_gemm_path(n, d, b, k):
     w = dg.single_layer(name="t", n_cache=n, n_query=b, dim=d, num_classes=9, dtype="bf16", sigma=0.6, k=k, seed=5)
