@@ -440,10 +440,18 @@ def run_reference(args):
             taus.append(float(np.float32(np.percentile(conf, p))))
         else:
             taus.append(float("inf"))
-    sample = args.cpu_sample or default_cpu_sample(w, reference_arm=True)
-    for _ in range(min(args.warmup, 1)):
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    if args.cpu_sample:
+        sample = args.cpu_sample
+    else:
+        # size the per-step sample from a short probe so that warm-up + K steps take about a minute
+        probe = min(8, w.stages[0].queries.shape[0])
+        t0 = time.perf_counter()
+        oracle_sample_step(w, taus, probe)
+        rate = probe / (time.perf_counter() - t0)
+        sample = int(max(1, min(w.stages[0].queries.shape[0], rate * 60.0 / (steps + warmup))))
+    for _ in range(warmup):
         oracle_sample_step(w, taus, sample)
-    steps = max(1, min(args.steps, 3))
     t0 = time.perf_counter()
     for _ in range(steps):
         oracle_sample_step(w, taus, sample)
@@ -451,7 +459,7 @@ def run_reference(args):
     cores = len(os.sched_getaffinity(0))
     value = sample * steps / dt
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
-            "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * dt / steps, "higher_is_better": True,
+            "warmup": warmup, "ms_per_step": 1e3 * dt / steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "stages": len(w.stages), "batch": sample, "k": w.k},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",

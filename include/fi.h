@@ -229,6 +229,14 @@ fi_status_t fi_cache_compute_threshold(fi_cache_t *cache, const void *val_acts, 
                                        const int32_t *model_labels, int64_t n, float *tau_out, int64_t *wrong_out,
                                        void *cuda_stream);
 
+/*
+ * Self-test of the failure path: enqueue a one-thread kernel that waits, with the given limit in SM cycles (at most
+ * 2e9, about a second), on a barrier that nothing completes.  The wait runs out, the kernel sets the cache's status
+ * word and returns; the next fi_cache_poll_status reports FI_ERR_TIMEOUT and the device stays usable.  Nothing
+ * faults, traps or hangs.
+ */
+fi_status_t fi_cache_selftest_wait(fi_cache_t *cache, int64_t limit_cycles, void *cuda_stream);
+
 /* Synchronise the device and return FI_ERR_TIMEOUT if a kernel of this cache gave up on a bounded wait
  * since the last poll (the word is cleared), FI_OK otherwise. */
 fi_status_t fi_cache_poll_status(fi_cache_t *cache);

@@ -23,7 +23,7 @@ FI_PATH_AUTO, FI_PATH_STREAM, FI_PATH_GEMM = 0, 1, 2
 EXPORTS = ["fi_cache_create", "fi_cache_destroy", "fi_cache_insert", "fi_cache_set_threshold", "fi_cache_set_path",
            "fi_cache_size", "fi_cache_lookup_batch", "fi_cascade_init", "fi_cascade_step", "fi_cache_lookup_batch_host",
            "fi_cascade_run_host", "fi_cache_poll_status", "fi_cache_set_profiling",
-           "fi_cache_read_profile", "fi_lookup_noalloc", "fi_cache_compute_threshold", "fi_cache_clear", "fi_kmeans_step", "fi_launch_count", "fi_last_error", "fi_status_string"]
+           "fi_cache_read_profile", "fi_lookup_noalloc", "fi_cache_compute_threshold", "fi_cache_clear", "fi_kmeans_step", "fi_cache_selftest_wait", "fi_launch_count", "fi_last_error", "fi_status_string"]
 
 
 class fi_cache_config_t(ctypes.Structure):
@@ -77,6 +77,7 @@ def load_library(path: Optional[str] = None):
     lib.fi_cascade_run_host.argtypes = [ctypes.POINTER(vp), i32, ctypes.POINTER(vp), i32, vp, vp, vp, vp, vp]
     lib.fi_cache_poll_status.argtypes = [vp]
     lib.fi_cache_clear.argtypes = [vp]
+    lib.fi_cache_selftest_wait.argtypes = [vp, i64, vp]
     lib.fi_kmeans_step.argtypes = [vp, vp, i64, vp, i64, vp, vp, vp, vp, vp, vp]
     lib.fi_cache_compute_threshold.argtypes = [vp, vp, i64, vp, i64, ctypes.POINTER(ctypes.c_float),
                                                ctypes.POINTER(i64), vp]
@@ -202,6 +203,11 @@ class FreezeCache:
 
     def poll_status(self) -> None:
         _check(self._lib.fi_cache_poll_status(self._h))
+
+    # -- fi_cache_selftest_wait
+    def selftest_wait(self, limit_cycles: int = 2_000_000) -> None:
+        """Enqueue the bounded-wait self-test; the next poll_status() raises FI_ERR_TIMEOUT."""
+        _check(self._lib.fi_cache_selftest_wait(self._h, int(limit_cycles), _stream_ptr(self.device)))
 
     # -- fi_cache_clear
     def clear(self) -> None:

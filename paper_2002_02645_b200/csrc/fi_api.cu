@@ -678,6 +678,15 @@ fi_status_t fi_cache_compute_threshold(fi_cache_t *c, const void *val_acts, int6
     return FI_OK;
 }
 
+fi_status_t fi_cache_selftest_wait(fi_cache_t *c, int64_t limit_cycles, void *cuda_stream) {
+    if (!c || limit_cycles < 1 || limit_cycles > 2000000000ll) {
+        set_error("fi_cache_selftest_wait: null cache or limit outside 1..2e9 cycles");
+        return FI_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(c->cfg.device);
+    return launch_wait_selftest(c, (long long)limit_cycles, static_cast<cudaStream_t>(cuda_stream));
+}
+
 fi_status_t fi_cache_poll_status(fi_cache_t *c) {
     if (!c) {
         set_error("fi_cache_poll_status: null cache");

@@ -81,7 +81,8 @@ __device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false (and raises the abort flag and the status word) when the limit is reached or
 // another thread of the CTA has already given up.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, SmemCtl *ctl, int32_t *status, int where) {
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, SmemCtl *ctl, int32_t *status, int where,
+                                          long long limit_cycles = kWaitLimitCycles) {
     if (mbar_try(bar, parity)) return true;
     // the SM's own cycle counter is a register read; the wait sits on the hand-over path of every stage and tile
     const long long t0 = clock64();
@@ -90,7 +91,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, SmemCt
         if (mbar_try(bar, parity)) return true;
         if ((++spins & 0xFF) == 0) {
             if (ctl->abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (clock64() - t0 > limit_cycles) {
                 ctl->abort_flag = 1;
                 atomicCAS(status, 0, (int32_t)(FI_ERR_TIMEOUT | (where << 8)));
                 return false;
@@ -715,6 +716,18 @@ tail_select_kernel(const GemmPlan *__restrict__ plan_dev, int num_ctas, const fl
     }
 }
 
+// Exercises the bounded wait on purpose: one thread waits on a barrier that nothing will ever complete, with a
+// short limit, and must come back with the status word set instead of hanging.
+__global__ void wait_selftest_kernel(long long limit_cycles, int32_t *status) {
+    __shared__ SmemCtl ctl;
+    if (threadIdx.x == 0) {
+        ctl.abort_flag = 0;
+        mbar_init(&ctl.full[0], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_wait(&ctl.full[0], 0, &ctl, status, 9, limit_cycles);
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -807,6 +820,12 @@ fi_status_t launch_msub(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, c
 // Query rows per CTA tile: 256 when the batch can fill it and a tile's k-loop is long enough (>= 32 k-blocks) to
 // dwarf the select that can no longer overlap it; 128 otherwise.
 int gemm_tile_m(int batch_max, int dim) { return (batch_max > kTileM && dim >= 32 * kBlockK) ? 2 * kTileM : kTileM; }
+
+fi_status_t launch_wait_selftest(fi_cache *c, long long limit_cycles, cudaStream_t stream) {
+    wait_selftest_kernel<<<1, 32, 0, stream>>>(limit_cycles, c->status_dev);
+    count_launch();
+    return check_launch("wait_selftest_kernel");
+}
 
 fi_status_t ensure_tensor_maps(fi_cache *c) {
     if (c->tmaps_ready) return FI_OK;

@@ -209,6 +209,7 @@ fi_status_t launch_kmeans_update(const fi_cache *c, const void *points, int64_t 
                                  const int32_t *assign, int64_t n, void *new_centres, int32_t *counts,
                                  int32_t *majority, float *fraction, cudaStream_t stream);
 
+fi_status_t launch_wait_selftest(fi_cache *c, long long limit_cycles, cudaStream_t stream);
 fi_status_t ensure_tensor_maps(fi_cache *c);
 size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, int dim);
 int gemm_tile_m(int batch_max, int dim);

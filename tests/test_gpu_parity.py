@@ -354,3 +354,21 @@ def test_compute_threshold_matches_oracle(path, max_batch):
     hit = out.hit.cpu().numpy() == 1
     assert hit.any() and (out.label.cpu().numpy()[hit] == model[:first][hit]).all()
     cache.close()
+
+
+# ------------------------------------------------------------------ failure path: a wait that runs out
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    w = dg.single_layer(name="t", n_cache=500, n_query=40, dim=128, num_classes=5, dtype="bf16", sigma=0.5, k=3, seed=17)
+    st = w.stages[0]
+    cache = make_cache(st, k=3, num_classes=5, tau=0.0, max_batch=40, path=fb.FI_PATH_GEMM)
+    before = run_lookup(cache, st.queries)
+    cache.selftest_wait(2_000_000)                       # about a millisecond on a barrier nothing completes
+    with pytest.raises(fb.FiError) as e:
+        cache.poll_status()
+    assert e.value.status == 6 and "bounded wait" in str(e.value)
+    cache.poll_status()                                   # the word was cleared by the poll that reported it
+    after = run_lookup(cache, st.queries)                 # same device, same context, same answers
+    for a, b in zip(before, after):
+        np.testing.assert_array_equal(a, b)
+    cache.close()
