@@ -524,13 +524,97 @@ def run_kmeans(args):
     cache.close()
 
 
+def run_rowshard(args):
+    """The 200,000-entry single-layer workload with the cache ROWS split over the ranks (strong scaling: the same
+    8,192 requests and the same entries at every N).  Every rank looks all requests up in its rows, one all-gather
+    moves batch x k x 16 bytes per rank, every rank merges and votes.  At N=1 this is the plain look-up plus the two
+    small kernels of the exchange."""
+    import torch
+    import torch.distributed as dist
+    from paper_2002_02645_b200 import binding as fb
+    from paper_2002_02645_b200 import build as fbuild
+    from paper_2002_02645_b200 import sharding
+    rank, local, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        fbuild.build_library()
+    if world > 1:
+        dist.barrier()
+    w = build_workload("cfg3", seed=0)
+    st = w.stages[0]
+    n, b0 = st.cache_vecs.shape[0], st.queries.shape[0]
+    lo, hi = sharding.shard_bounds(n, world, rank)
+    cache = fb.FreezeCache(dim=st.dim, capacity=hi - lo, num_classes=w.num_classes, k=w.k, dtype=fb.FI_BF16, device=local,
+                           max_batch=max(b0, st.calib.shape[0]))
+    rows = max(1, (512 << 20) // (st.dim * 2))
+    for a in range(lo, hi, rows):
+        b = min(hi, a + rows)
+        cache.insert(to_dev(st.cache_vecs[a:b], dev), torch.from_numpy(st.cache_labels[a:b]).to(dev))
+    cache.set_threshold(0.0)
+    conf = sharding.sharded_lookup(cache, to_dev(st.calib, dev), lo).conf.cpu().numpy().astype(np.float64)
+    tau = float(np.float32(np.percentile(conf[np.isfinite(conf)], w.meta["percentiles"][0])))
+    cache.set_threshold(tau)
+    q = to_dev(st.queries, dev)
+
+    def fence():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        out = sharding.sharded_lookup(cache, q, lo)
+    fence()
+    cache.poll_status()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    l0 = fb.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    fence()
+    e0.record()
+    for _ in range(args.steps):
+        out = sharding.sharded_lookup(cache, q, lo)
+    e1.record()
+    fence()
+    launches = fb.launch_count() - l0
+    clocks = sampler.stop()
+    cache.poll_status()
+    ms_total, _ = sharding.reduce_timing(e0.elapsed_time(e1), 0, dev)
+    ms = ms_total / args.steps
+    if rank == 0:
+        peaks, src = load_peaks()
+        tf = 2.0 * b0 * n * st.dim / (ms * 1e-3) / 1e12 / world          # per GPU, whole step as the duration
+        print(json.dumps({"metric": METRIC, "value": b0 / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+                          "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+                          "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "bf16",
+                          "data": "synthetic",
+                          "config": {"workload": w.name + "_row_sharded", "batch": b0, "entries": n, "dim": st.dim,
+                                     "k": w.k, "rows_per_rank": hi - lo, "exchange_bytes_per_rank": b0 * w.k * 16,
+                                     "hit_rate": float(out.hit.float().mean().item()),
+                                     "l2": "inputs larger than L2"},
+                          "gpu_launches": launches, "clocks": clocks,
+                          "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops_sustained"],
+                                       "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops_sustained"],
+                                       "peak_source": f"cuBLAS bf16 sustained, {src}; whole step as the duration",
+                                       "traffic": None}}))
+    cache.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0", "kmeans"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0", "kmeans", "cfg3-rows"])
     ap.add_argument("--cpu-sample", type=int, default=0,
                     help="requests per oracle timing (0: sized for 10-30 s of CPU work)")
     ap.add_argument("--batch", type=int, default=16, help="batch of the latency workload (cfg5): 1, 4 or 16")
@@ -539,6 +623,8 @@ def main():
     args = ap.parse_args()
     if args.workload == "kmeans":
         run_kmeans(args)
+    elif args.workload == "cfg3-rows" and args.impl == "ours":
+        run_rowshard(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -230,6 +230,22 @@ fi_status_t fi_cache_compute_threshold(fi_cache_t *cache, const void *val_acts, 
                                        void *cuda_stream);
 
 /*
+ * Cache rows sharded over several GPUs (the paper has one cache per layer on one machine; with entries split over
+ * ranks, rank g holding global rows [offset_g, offset_g + size_g), the k nearest of the whole cache are among
+ * the k nearest of every shard).  Step 1, on each rank after fi_cache_lookup_batch with topk outputs:
+ * fi_cache_neighbor_tuples turns its neighbour indices [n = batch*k] into travelling tuples: global index
+ * (local + index_offset, -1 stays -1), label and weight of each neighbour.  Step 2, after the ranks exchanged their
+ * tuples and distances (e.g. one all-gather): fi_merge_shard_lookups merges [shards][batch][k] tuples per query
+ * by (distance, global index), keeps k, and applies the vote and hit rule of Sec. 3 / Pseudocode 1 exactly as
+ * fi_cache_lookup_batch does.  All pointers are device pointers on the current device; asynchronous.
+ */
+fi_status_t fi_cache_neighbor_tuples(const fi_cache_t *cache, const int32_t *topk_idx, int64_t n, int32_t index_offset,
+                                     int32_t *global_idx, int32_t *label, float *weight, void *cuda_stream);
+fi_status_t fi_merge_shard_lookups(int32_t shards, int32_t batch, int32_t k, const float *dist, const int32_t *global_idx,
+                                   const int32_t *label, const float *weight, int32_t metric, int32_t rule,
+                                   float threshold, const fi_lookup_out_t *out, void *cuda_stream);
+
+/*
  * Self-test of the failure path: enqueue a one-thread kernel that waits, with the given limit in SM cycles (at most
  * 2e9, about a second), on a barrier that nothing completes.  The wait runs out, the kernel sets the cache's status
  * word and returns; the next fi_cache_poll_status reports FI_ERR_TIMEOUT and the device stays usable.  Nothing

@@ -190,6 +190,35 @@ def kmeans_step(points: np.ndarray, centres: np.ndarray, point_labels: np.ndarra
     return KMeansStep(assign, new, counts, majority, fraction)
 
 
+def merge_shards(shard_results: Sequence[LookupResult], shard_offsets: Sequence[int],
+                 shard_labels: Sequence[np.ndarray], *, k: int, tau: float, rule: int = RULE_CONF_GT,
+                 metric: int = METRIC_SQL2, shard_weights: Optional[Sequence[Optional[np.ndarray]]] = None) -> LookupResult:
+    """Look-up against a cache whose rows are split into shards, from the shards' own look-up results: per query the
+    shards' neighbour tuples are pooled under global row numbers, the k smallest under (D, n) kept, and the vote of
+    Sec. 3 applied to them."""
+    batch = shard_results[0].ni.shape[0]
+    res = LookupResult(np.empty(batch, np.int32), np.empty(batch, np.float64), np.empty(batch, np.uint8),
+                       np.full((batch, k), np.inf), np.full((batch, k), -1, np.int64), np.full(batch, np.inf))
+    for b in range(batch):
+        pool = []
+        for s, r in enumerate(shard_results):
+            for j in range(r.ni.shape[1]):
+                li = int(r.ni[b, j])
+                if li >= 0:
+                    w = 1.0 if shard_weights is None or shard_weights[s] is None else float(shard_weights[s][li])
+                    pool.append((float(r.nd[b, j]), li + int(shard_offsets[s]), int(shard_labels[s][li]), w))
+        pool.sort(key=lambda t: (t[0], t[1]))
+        top = pool[:k]
+        lab, conf, hit = vote([t[0] for t in top], [t[2] for t in top], [t[3] for t in top], metric=metric, rule=rule,
+                              tau=tau) if top else (-1, 0.0, False)
+        res.label[b], res.conf[b], res.hit[b] = lab, conf, int(hit)
+        for j, t in enumerate(top):
+            res.nd[b, j], res.ni[b, j] = t[0], t[1]
+        if len(pool) > k:
+            res.next_d[b] = pool[k][0]
+    return res
+
+
 def compact(active: np.ndarray, hit: np.ndarray) -> np.ndarray:
     """Ids of `active` whose look-up missed, order kept (Sec. 5, batch reconstruction)."""
     a = np.ascontiguousarray(active, dtype=np.int32)

@@ -23,7 +23,7 @@ FI_PATH_AUTO, FI_PATH_STREAM, FI_PATH_GEMM = 0, 1, 2
 EXPORTS = ["fi_cache_create", "fi_cache_destroy", "fi_cache_insert", "fi_cache_set_threshold", "fi_cache_set_path",
            "fi_cache_size", "fi_cache_lookup_batch", "fi_cascade_init", "fi_cascade_step", "fi_cache_lookup_batch_host",
            "fi_cascade_run_host", "fi_cache_poll_status", "fi_cache_set_profiling",
-           "fi_cache_read_profile", "fi_lookup_noalloc", "fi_cache_compute_threshold", "fi_cache_clear", "fi_kmeans_step", "fi_cache_selftest_wait", "fi_launch_count", "fi_last_error", "fi_status_string"]
+           "fi_cache_read_profile", "fi_lookup_noalloc", "fi_cache_compute_threshold", "fi_cache_clear", "fi_kmeans_step", "fi_cache_selftest_wait", "fi_cache_neighbor_tuples", "fi_merge_shard_lookups", "fi_launch_count", "fi_last_error", "fi_status_string"]
 
 
 class fi_cache_config_t(ctypes.Structure):
@@ -77,6 +77,9 @@ def load_library(path: Optional[str] = None):
     lib.fi_cascade_run_host.argtypes = [ctypes.POINTER(vp), i32, ctypes.POINTER(vp), i32, vp, vp, vp, vp, vp]
     lib.fi_cache_poll_status.argtypes = [vp]
     lib.fi_cache_clear.argtypes = [vp]
+    lib.fi_cache_neighbor_tuples.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
+    lib.fi_merge_shard_lookups.argtypes = [i32, i32, i32, vp, vp, vp, vp, i32, i32, ctypes.c_float,
+                                           ctypes.POINTER(fi_lookup_out_t), vp]
     lib.fi_cache_selftest_wait.argtypes = [vp, i64, vp]
     lib.fi_kmeans_step.argtypes = [vp, vp, i64, vp, i64, vp, vp, vp, vp, vp, vp]
     lib.fi_cache_compute_threshold.argtypes = [vp, vp, i64, vp, i64, ctypes.POINTER(ctypes.c_float),
@@ -194,6 +197,7 @@ class FreezeCache:
     # -- fi_cache_set_threshold / fi_cache_set_path / fi_cache_size / fi_cache_poll_status
     def set_threshold(self, tau: float) -> None:
         _check(self._lib.fi_cache_set_threshold(self._h, float(tau)))
+        self.cfg.threshold = float(tau)
 
     def set_path(self, path: int) -> None:
         _check(self._lib.fi_cache_set_path(self._h, int(path)))
@@ -203,6 +207,17 @@ class FreezeCache:
 
     def poll_status(self) -> None:
         _check(self._lib.fi_cache_poll_status(self._h))
+
+    # -- fi_cache_neighbor_tuples
+    def neighbor_tuples(self, topk_idx: torch.Tensor, index_offset: int):
+        """(global index, label, weight) of the neighbours a look-up on this shard returned."""
+        n = topk_idx.numel()
+        gi = torch.empty_like(topk_idx)
+        lab = torch.empty_like(topk_idx)
+        wgt = torch.empty(topk_idx.shape, dtype=torch.float32, device=self.device)
+        _check(self._lib.fi_cache_neighbor_tuples(self._h, _dp(topk_idx), n, int(index_offset), _dp(gi), _dp(lab), _dp(wgt),
+                                                  _stream_ptr(self.device)))
+        return gi, lab, wgt
 
     # -- fi_cache_selftest_wait
     def selftest_wait(self, limit_cycles: int = 2_000_000) -> None:
@@ -296,6 +311,19 @@ def lookup_noalloc(cache_vecs: torch.Tensor, labels: torch.Tensor, weights: torc
                                                 cache_vecs.shape[1], dtype, k, rule, metric, float(threshold),
                                                 _dp(queries), queries.stride(0), queries.shape[0], ctypes.byref(st),
                                                 _stream_ptr(dev)))
+    return out
+
+
+def merge_shard_lookups(dist: torch.Tensor, global_idx: torch.Tensor, label: torch.Tensor, weight: torch.Tensor, *,
+                        metric: int = FI_METRIC_SQL2, rule: int = FI_HIT_CONF_GT, threshold: float = 0.0) -> LookupOut:
+    """fi_merge_shard_lookups on gathered tuples of shape [shards, batch, k]."""
+    shards, batch, k = dist.shape
+    out = LookupOut(batch, k, dist.device)
+    st = out.as_struct()
+    with torch.cuda.device(dist.device):
+        _check(load_library().fi_merge_shard_lookups(shards, batch, k, _dp(dist.contiguous()), _dp(global_idx.contiguous()),
+                                                     _dp(label.contiguous()), _dp(weight.contiguous()), metric, rule,
+                                                     float(threshold), ctypes.byref(st), _stream_ptr(dist.device)))
     return out
 
 

@@ -678,6 +678,30 @@ fi_status_t fi_cache_compute_threshold(fi_cache_t *c, const void *val_acts, int6
     return FI_OK;
 }
 
+fi_status_t fi_cache_neighbor_tuples(const fi_cache_t *c, const int32_t *topk_idx, int64_t n, int32_t index_offset,
+                                     int32_t *global_idx, int32_t *label, float *weight, void *cuda_stream) {
+    if (!c || n < 0 || (n > 0 && (!topk_idx || !global_idx || !label || !weight))) {
+        set_error("fi_cache_neighbor_tuples: null or negative argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(c->cfg.device);
+    return launch_neighbor_tuples(c, topk_idx, n, index_offset, global_idx, label, weight,
+                                  static_cast<cudaStream_t>(cuda_stream));
+}
+
+fi_status_t fi_merge_shard_lookups(int32_t shards, int32_t batch, int32_t k, const float *dist, const int32_t *global_idx,
+                                   const int32_t *label, const float *weight, int32_t metric, int32_t rule,
+                                   float threshold, const fi_lookup_out_t *out, void *cuda_stream) {
+    if (shards < 1 || batch < 0 || k < 1 || k > kMaxK || !out ||
+        (batch > 0 && (!dist || !global_idx || !label || !weight || !out->label || !out->conf || !out->hit)) ||
+        (rule != FI_HIT_CONF_GT && rule != FI_HIT_DIST_LE) || (metric != FI_METRIC_SQL2 && metric != FI_METRIC_L2)) {
+        set_error("fi_merge_shard_lookups: invalid argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    return launch_merge_vote(shards, batch, k, dist, global_idx, label, weight, metric, rule, threshold, *out,
+                             static_cast<cudaStream_t>(cuda_stream));
+}
+
 fi_status_t fi_cache_selftest_wait(fi_cache_t *c, int64_t limit_cycles, void *cuda_stream) {
     if (!c || limit_cycles < 1 || limit_cycles > 2000000000ll) {
         set_error("fi_cache_selftest_wait: null cache or limit outside 1..2e9 cycles");

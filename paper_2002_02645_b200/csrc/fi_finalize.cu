@@ -308,7 +308,113 @@ __global__ void wrong_max_kernel(const int32_t *__restrict__ label, const float 
     }
 }
 
+// Cache rows sharded over several GPUs: each shard answers a look-up with its own k nearest entries (exact distances).
+// neighbor_tuples_kernel turns a shard's neighbour indices into tuples that can travel: global index, label, weight.
+__global__ void neighbor_tuples_kernel(const int32_t *__restrict__ topk_idx, int64_t n, int32_t index_offset,
+                                       const int32_t *__restrict__ labels, const float *__restrict__ weights,
+                                       int32_t *__restrict__ out_idx, int32_t *__restrict__ out_label,
+                                       float *__restrict__ out_weight) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t li = topk_idx[i];
+        out_idx[i] = li < 0 ? -1 : li + index_offset;
+        out_label[i] = li < 0 ? -1 : labels[li];
+        out_weight[i] = li < 0 ? 0.f : weights[li];
+    }
+}
+
+// merge_vote_kernel: one thread per query merges the shards' tuples [shard][query][k] by (distance, global index),
+// keeps the k nearest and applies the same vote and hit rule as finalize_kernel.  Every rank runs it on the same
+// gathered tuples and gets the same answer.
+__global__ void merge_vote_kernel(int shards, int batch, int k, const float *__restrict__ dist,
+                                  const int32_t *__restrict__ idx, const int32_t *__restrict__ label,
+                                  const float *__restrict__ weight, int metric, int rule, float tau,
+                                  int32_t *__restrict__ out_label, float *__restrict__ out_conf,
+                                  uint8_t *__restrict__ out_hit, float *__restrict__ out_dist,
+                                  int32_t *__restrict__ out_idx) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= batch) return;
+    const float kInf = __int_as_float(0x7F800000);
+    float bd[kMaxK];
+    int32_t bi[kMaxK], bl[kMaxK];
+    float bw[kMaxK];
+    int have = 0;
+    for (int s = 0; s < shards; ++s) {
+        const int64_t base = ((int64_t)s * batch + b) * k;
+        for (int j = 0; j < k; ++j) {
+            const int32_t gi = idx[base + j];
+            if (gi < 0) continue;
+            const float d = dist[base + j];
+            if (have == k && !pair_less(d, gi, bd[k - 1], bi[k - 1])) continue;
+            int pos = have < k ? have : k - 1;
+            while (pos > 0 && pair_less(d, gi, bd[pos - 1], bi[pos - 1])) {
+                bd[pos] = bd[pos - 1];
+                bi[pos] = bi[pos - 1];
+                bl[pos] = bl[pos - 1];
+                bw[pos] = bw[pos - 1];
+                --pos;
+            }
+            bd[pos] = d;
+            bi[pos] = gi;
+            bl[pos] = label[base + j];
+            bw[pos] = weight[base + j];
+            if (have < k) ++have;
+        }
+    }
+    const int k_eff = have;
+    int32_t best_label = -1;
+    float best_c = 0.f, best_dwin = 0.f;
+    int best_m = 0;
+    for (int a = 0; a < k_eff; ++a) {
+        bool seen = false;
+        for (int e = 0; e < a; ++e) seen |= (bl[e] == bl[a]);
+        if (seen) continue;
+        int m = 0;
+        float sum = 0.f;
+        for (int j = a; j < k_eff; ++j) {
+            if (bl[j] != bl[a]) continue;
+            const float dj = metric == FI_METRIC_L2 ? sqrtf(bd[j]) : bd[j];
+            sum += bw[j] / dj;
+            ++m;
+        }
+        const float c = ((float)m / (float)k_eff) * sum;
+        if (best_label < 0 || c > best_c || (c == best_c && m > best_m)) {
+            best_label = bl[a];
+            best_c = c;
+            best_m = m;
+            best_dwin = metric == FI_METRIC_L2 ? sqrtf(bd[a]) : bd[a];
+        }
+    }
+    const bool hit = k_eff > 0 && (rule == FI_HIT_CONF_GT ? best_c > tau : best_dwin <= tau);
+    out_label[b] = best_label;
+    out_conf[b] = best_c;
+    out_hit[b] = hit ? 1 : 0;
+    if (out_dist)
+        for (int j = 0; j < k; ++j) out_dist[(int64_t)b * k + j] = j < k_eff ? bd[j] : kInf;
+    if (out_idx)
+        for (int j = 0; j < k; ++j) out_idx[(int64_t)b * k + j] = j < k_eff ? bi[j] : -1;
+}
+
 }  // namespace
+
+fi_status_t launch_neighbor_tuples(const fi_cache *c, const int32_t *topk_idx, int64_t n, int32_t index_offset,
+                                   int32_t *out_idx, int32_t *out_label, float *out_weight, cudaStream_t stream) {
+    if (n <= 0) return FI_OK;
+    int grid = (int)((n + 255) / 256 < 2048 ? (n + 255) / 256 : 2048);
+    neighbor_tuples_kernel<<<grid, 256, 0, stream>>>(topk_idx, n, index_offset, c->labels, c->weights, out_idx, out_label,
+                                                     out_weight);
+    count_launch();
+    return check_launch("neighbor_tuples_kernel");
+}
+
+fi_status_t launch_merge_vote(int shards, int batch, int k, const float *dist, const int32_t *idx, const int32_t *label,
+                              const float *weight, int metric, int rule, float tau, const fi_lookup_out_t &out,
+                              cudaStream_t stream) {
+    if (batch <= 0) return FI_OK;
+    merge_vote_kernel<<<(batch + 127) / 128, 128, 0, stream>>>(shards, batch, k, dist, idx, label, weight, metric, rule, tau,
+                                                              out.label, out.conf, out.hit, out.topk_dist, out.topk_idx);
+    count_launch();
+    return check_launch("merge_vote_kernel");
+}
 
 fi_status_t launch_wrong_max(const int32_t *label, const float *conf, const int32_t *ref, int32_t n, int32_t *acc,
                              cudaStream_t stream) {

@@ -209,6 +209,11 @@ fi_status_t launch_kmeans_update(const fi_cache *c, const void *points, int64_t 
                                  const int32_t *assign, int64_t n, void *new_centres, int32_t *counts,
                                  int32_t *majority, float *fraction, cudaStream_t stream);
 
+fi_status_t launch_neighbor_tuples(const fi_cache *c, const int32_t *topk_idx, int64_t n, int32_t index_offset,
+                                   int32_t *out_idx, int32_t *out_label, float *out_weight, cudaStream_t stream);
+fi_status_t launch_merge_vote(int shards, int batch, int k, const float *dist, const int32_t *idx, const int32_t *label,
+                              const float *weight, int metric, int rule, float tau, const fi_lookup_out_t &out,
+                              cudaStream_t stream);
 fi_status_t launch_wait_selftest(fi_cache *c, long long limit_cycles, cudaStream_t stream);
 fi_status_t ensure_tensor_maps(fi_cache *c);
 size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, int dim);

@@ -372,3 +372,35 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     for a, b in zip(before, after):
         np.testing.assert_array_equal(a, b)
     cache.close()
+
+
+# ------------------------------------------------------------------ cache rows split over several caches (shards)
+
+@pytest.mark.parametrize("path", [fb.FI_PATH_GEMM, fb.FI_PATH_STREAM])
+def test_row_sharded_lookup_matches_unsharded_oracle(path):
+    """Three shards stand in for three GPUs: each answers from its rows, the tuples are pooled as an all-gather would
+    deliver them, and every "rank" merges them with fi_merge_shard_lookups."""
+    from paper_2002_02645_b200.datagen import StageData
+    w = dg.single_layer(name="t", n_cache=3000, n_query=96, dim=512, num_classes=6, dtype="bf16", sigma=0.5, k=5, seed=25)
+    st = w.stages[0]
+    ref0 = fo.lookup(st.queries, st.cache_vecs, st.cache_labels, k=5, tau=0.0)
+    tau = f32(np.median(ref0.conf))
+    ref = fo.lookup(st.queries, st.cache_vecs, st.cache_labels, k=5, tau=tau)
+    cuts = [0, 1000, 1003, 3000]
+    q = to_device(st.queries)
+    gathered = [[], [], [], []]
+    for a, b in zip(cuts, cuts[1:]):
+        shard = StageData(st.dim, "bf16", st.cache_vecs[a:b], st.cache_labels[a:b], st.queries)
+        c = make_cache(shard, k=5, num_classes=6, tau=tau, max_batch=96, path=path)
+        out = c.lookup_batch(q)
+        gi, lab, wgt = c.neighbor_tuples(out.topk_idx, a)
+        torch.cuda.synchronize()
+        for lst, t in zip(gathered, (out.topk_dist, gi, lab, wgt)):
+            lst.append(t.clone())
+        c.close()
+    merged = fb.merge_shard_lookups(*[torch.stack(g) for g in gathered], threshold=tau)
+    torch.cuda.synchronize()
+    compare_lookup(merged.label.cpu().numpy(), merged.conf.cpu().numpy(), merged.hit.cpu().numpy(),
+                   merged.topk_dist.cpu().numpy(), merged.topk_idx.cpu().numpy(), ref, storage="bf16", tau=tau, rule=0,
+                   cache_labels=st.cache_labels)
+    assert 0 < ref.hit.sum() < 96

@@ -64,3 +64,47 @@ def test_two_ranks_gloo(tmp_path):
     port = _free_port()
     mp.spawn(_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
     assert (tmp_path / "result").read_text() == "ok"
+
+
+def _row_shard_worker(rank, world, port, out_dir):
+    """Cache rows split over two ranks: each rank looks the whole batch up in its rows (oracle), the neighbour tuples
+    travel through the one all-gather the GPU path uses, and the merge of what arrived equals the unsharded answer."""
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from oracle import fi_oracle as fo
+    from paper_2002_02645_b200 import datagen as dg
+    fo.set_threads(1)
+    st = dg.single_layer(name="t", n_cache=333, n_query=24, dim=64, num_classes=5, dtype="f32", sigma=0.5, k=4,
+                         seed=31).stages[0]
+    cuts = [sharding.shard_bounds(333, world, r) for r in range(world)]
+    lo, hi = cuts[rank]
+    mine = fo.lookup(st.queries, st.cache_vecs[lo:hi], st.cache_labels[lo:hi], k=4, tau=0.46)
+    tensors = [torch.from_numpy(mine.nd.astype(np.float32)),
+               torch.from_numpy((mine.ni + lo).astype(np.int32)),
+               torch.from_numpy(st.cache_labels[lo:hi][mine.ni].astype(np.int32)),
+               torch.ones(mine.ni.shape, dtype=torch.float32)]
+    d, gi, lab, wgt = sharding.gather_shard_tuples(tensors)
+    ok = d.shape == (world, 24, 4) and d.dtype == torch.float32 and gi.dtype == torch.int32
+    ok = ok and torch.equal(d[rank], tensors[0]) and torch.equal(gi[rank], tensors[1])
+    # every rank holds every shard's tuples now; rebuild per-shard results from them and merge
+    parts = []
+    for r, (a, b) in enumerate(cuts):
+        nd = d[r].numpy().astype(np.float64)
+        parts.append(fo.LookupResult(None, None, None, nd, gi[r].numpy().astype(np.int64) - a, None))
+        ok = ok and np.array_equal(lab[r].numpy(), st.cache_labels[gi[r].numpy()])
+    merged = fo.merge_shards(parts, [a for a, _ in cuts], [st.cache_labels[a:b] for a, b in cuts], k=4, tau=0.46)
+    whole = fo.lookup(st.queries, st.cache_vecs, st.cache_labels, k=4, tau=0.46)
+    ok = ok and np.array_equal(merged.ni, whole.ni) and np.array_equal(merged.label, whole.label) \
+        and np.array_equal(merged.hit, whole.hit) and 0 < whole.hit.sum() < 24
+    with open(os.path.join(out_dir, f"result{rank}"), "w") as f:
+        f.write("ok" if ok else "bad")
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_row_sharding_two_ranks_gloo(tmp_path):
+    from oracle import fi_oracle as fo
+    fo.build()
+    port = _free_port()
+    mp.spawn(_row_shard_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    assert (tmp_path / "result0").read_text() == "ok" and (tmp_path / "result1").read_text() == "ok"

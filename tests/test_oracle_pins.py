@@ -435,3 +435,20 @@ def test_kmeans_step_against_sklearn_and_invariants():
     # (Sec. 2.1's observation on cluster purity)
     live = st.counts > 0
     assert (st.fraction[live] >= 1.0 / 6).all() and (st.fraction[live] <= 1.0).all() and (st.fraction[live] > 0.95).any()
+
+
+# ------------------------------------------------------------------ cache rows split into shards
+
+def test_merge_of_row_shards_equals_the_unsharded_lookup():
+    x, q, lab = _small_case(seed=23, n=301, b=40, c=5)
+    w = np.random.default_rng(24).uniform(0.5, 1.0, 301).astype(np.float32)
+    whole = fo.lookup(q, x, lab, k=4, tau=0.03, weights=w)
+    cuts = [0, 100, 101, 250, 301]                                    # uneven shards, one of a single row
+    parts = [fo.lookup(q, x[a:b], lab[a:b], k=4, tau=0.03, weights=w[a:b]) for a, b in zip(cuts, cuts[1:])]
+    merged = fo.merge_shards(parts, cuts[:-1], [lab[a:b] for a, b in zip(cuts, cuts[1:])], k=4, tau=0.03,
+                             shard_weights=[w[a:b] for a, b in zip(cuts, cuts[1:])])
+    np.testing.assert_array_equal(merged.ni, whole.ni)
+    np.testing.assert_array_equal(merged.nd, whole.nd)
+    np.testing.assert_array_equal(merged.label, whole.label)
+    np.testing.assert_array_equal(merged.conf, whole.conf)
+    np.testing.assert_array_equal(merged.hit, whole.hit)
