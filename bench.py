@@ -542,18 +542,100 @@ def run_kmeans(args):
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / args.steps
+    # the point of the k-means cache (Sec. 4, Table 1): a look-up against 200 tagged centres instead of 40,000 points
+    centres, counts, major, frac = cache.kmeans_step(pts, labs)[1:5]
+    km = fb.FreezeCache(dim=d, capacity=clusters, num_classes=10, k=1, dtype=fb.FI_BF16, max_batch=1024)
+    keep = counts > 0
+    km.insert(centres[keep].contiguous(), major[keep].contiguous(), frac[keep].contiguous())
+    full = fb.FreezeCache(dim=d, capacity=n, num_classes=10, k=1, dtype=fb.FI_BF16, max_batch=1024)
+    full.insert(pts, labs)
+    reqs = to_dev(dg.single_layer(name="q", n_cache=8, n_query=1024, dim=d, num_classes=10, dtype="bf16", sigma=0.5, k=1,
+                                  seed=0, query_seed=7).stages[0].queries, dev)
+    lookup_ms = {}
+    for name, cc in (("kmeans_cache_200", km), ("full_cache_40000", full)):
+        out = fb.LookupOut(1024, 1, dev, with_topk=False)
+        for _ in range(3):
+            cc.lookup_batch(reqs, out=out)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.steps):
+            cc.lookup_batch(reqs, out=out)
+        b.record()
+        torch.cuda.synchronize()
+        lookup_ms[name] = a.elapsed_time(b) / args.steps
+    km.close()
+    full.close()
     peaks, src = load_peaks()
     nbytes = 2.0 * n * d * 2          # the points are read once by the assignment and once by the update
     print(json.dumps({"metric": "k-means Lloyd iteration, points/s", "value": n / (ms * 1e-3), "unit": "points/s",
                       "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
                       "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
                       "config": {"workload": w.name, "points": n, "dim": d, "clusters": clusters,
-                                 "l2": "points (82 MB) fit in L2: figures are L2-warm"},
+                                 "l2": "points (82 MB) fit in L2: figures are L2-warm",
+                                 "lookup_ms_batch_1024": lookup_ms},
                       "gpu_launches": fb.launch_count() - l0,
                       "roofline": {"bound": "hbm", "achieved": nbytes / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                                    "unit": "GB/s", "frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                    "peak_source": f"copy bandwidth, {src}", "traffic": None}}))
     cache.close()
+
+
+def run_tau_sweep(args):
+    """Frozen share against agreement with the request's class as the thresholds move (the axes of the paper's
+    threshold study, Sec. 5), on the 4-stage synthetic cascade: every stage's threshold is set to the p-th percentile
+    of the library's confidences on the calibration batch, p swept; one more point uses ComputeThresholds (Pseudocode 1)
+    with the calibration requests' classes standing in for the model's predictions."""
+    import torch
+    from paper_2002_02645_b200 import binding as fb
+    from paper_2002_02645_b200 import build as fbuild
+    fbuild.build_library()
+    dev = torch.device("cuda", 0)
+    w = build_workload("cfg2", seed=0)
+    b0, n_stage = w.stages[0].queries.shape[0], len(w.stages)
+    caches, acts, calib_conf = [], [], []
+    for st in w.stages:
+        c = fb.FreezeCache(dim=st.dim, capacity=st.cache_vecs.shape[0], num_classes=w.num_classes, k=w.k, dtype=fb.FI_BF16,
+                           max_batch=max(b0, st.calib.shape[0]))
+        c.insert(to_dev(st.cache_vecs, dev), torch.from_numpy(st.cache_labels).to(dev))
+        c.set_threshold(0.0)
+        conf = c.lookup_batch(to_dev(st.calib, dev), with_topk=False).conf.cpu().numpy().astype(np.float64)
+        calib_conf.append(conf[np.isfinite(conf)])
+        caches.append(c)
+        acts.append(to_dev(st.queries, dev))
+    state = fb.CascadeState(b0, dev)
+    classes = w.query_classes.astype(np.int64)
+
+    def run(taus):
+        for c, t in zip(caches, taus):
+            c.set_threshold(float(t))
+        fb.cascade_init(state, n_stage)
+        for l in range(n_stage):
+            fb.cascade_step(caches[l], acts[l], state, l)
+        torch.cuda.synchronize()
+        stage = state.exit_stage.cpu().numpy()[:b0]
+        label = state.final_label.cpu().numpy()[:b0]
+        frozen = stage < n_stage
+        return {"thresholds": [float(t) for t in taus], "frozen_share": float(frozen.mean()),
+                "frozen_by_stage": [int((stage == l).sum()) for l in range(n_stage)],
+                "agreement_of_frozen": float((label[frozen] == classes[frozen]).mean()) if frozen.any() else None}
+
+    points = []
+    for p in (5, 10, 20, 30, 40, 50, 60, 70, 80, 90, 95, 99):
+        r = run([np.float32(np.percentile(cc, p)) for cc in calib_conf])
+        r["percentile"] = p
+        points.append(r)
+    computed = []
+    for c, st in zip(caches, w.stages):
+        tau, wrong = c.compute_threshold(to_dev(st.calib, dev), torch.from_numpy(w.calib_classes.astype(np.int32)).to(dev))
+        computed.append({"tau": tau, "wrong_lookups": wrong})
+    r = run([x["tau"] for x in computed])
+    r["rule"] = "ComputeThresholds"
+    r["wrong_lookups_on_calibration"] = [x["wrong_lookups"] for x in computed]
+    print(json.dumps({"study": "threshold sweep", "config": {"workload": w.name, "batch": b0, "stages": n_stage},
+                      "data": "synthetic", "points": points, "compute_thresholds": r}))
+    for c in caches:
+        c.close()
 
 
 def run_rowshard(args):
@@ -646,7 +728,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0", "kmeans", "cfg3-rows"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0", "kmeans", "cfg3-rows", "tau-sweep"])
     ap.add_argument("--cpu-sample", type=int, default=0,
                     help="requests per oracle timing (0: sized for 10-30 s of CPU work)")
     ap.add_argument("--batch", type=int, default=16, help="batch of the latency workload (cfg5): 1, 4 or 16")
@@ -655,6 +737,8 @@ def main():
     args = ap.parse_args()
     if args.workload == "kmeans":
         run_kmeans(args)
+    elif args.workload == "tau-sweep":
+        run_tau_sweep(args)
     elif args.workload == "cfg3-rows" and args.impl == "ours":
         run_rowshard(args)
     elif args.impl == "reference":

@@ -136,7 +136,8 @@ fi_status_t fi_cache_clear(fi_cache_t *cache);
  * Update step: per cluster the mean of its points, rounded to the cache's dtype; the number of points; the most
  * frequent of the points' labels (smaller label on ties) and its share.  A cluster without points keeps its
  * centre and gets label -1, share 0.
- *   points [n x ld_elems] device, dtype of the cache; point_labels [n] device int32 in [0, num_classes)
+ *   points [n x ld_elems] device, dtype of the cache; point_labels [n] device int32 in [0, num_classes) (a label
+ *   outside that range is left out of the majority count)
  *   assign_out [n] device int32; new_centres [size x dim] device, cache dtype; counts / majority_label [size]
  *   device int32; fraction [size] device float
  * Feeding (new_centres, majority_label, fraction) to fi_cache_clear + fi_cache_insert (as vecs, labels, weights)

@@ -310,12 +310,13 @@ __global__ void wrong_max_kernel(const int32_t *__restrict__ label, const float 
 
 // Cache rows sharded over several GPUs: each shard answers a look-up with its own k nearest entries (exact distances).
 // neighbor_tuples_kernel turns a shard's neighbour indices into tuples that can travel: global index, label, weight.
-__global__ void neighbor_tuples_kernel(const int32_t *__restrict__ topk_idx, int64_t n, int32_t index_offset,
-                                       const int32_t *__restrict__ labels, const float *__restrict__ weights,
+__global__ void neighbor_tuples_kernel(const int32_t *__restrict__ topk_idx, int64_t n, int64_t size,
+                                       int32_t index_offset, const int32_t *__restrict__ labels, const float *__restrict__ weights,
                                        int32_t *__restrict__ out_idx, int32_t *__restrict__ out_label,
                                        float *__restrict__ out_weight) {
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-        const int32_t li = topk_idx[i];
+        int32_t li = topk_idx[i];
+        if (li >= size) li = -1;   // not an index of this shard: treated as "no neighbour"
         out_idx[i] = li < 0 ? -1 : li + index_offset;
         out_label[i] = li < 0 ? -1 : labels[li];
         out_weight[i] = li < 0 ? 0.f : weights[li];
@@ -400,7 +401,7 @@ fi_status_t launch_neighbor_tuples(const fi_cache *c, const int32_t *topk_idx, i
                                    int32_t *out_idx, int32_t *out_label, float *out_weight, cudaStream_t stream) {
     if (n <= 0) return FI_OK;
     int grid = (int)((n + 255) / 256 < 2048 ? (n + 255) / 256 : 2048);
-    neighbor_tuples_kernel<<<grid, 256, 0, stream>>>(topk_idx, n, index_offset, c->labels, c->weights, out_idx, out_label,
+    neighbor_tuples_kernel<<<grid, 256, 0, stream>>>(topk_idx, n, c->size, index_offset, c->labels, c->weights, out_idx, out_label,
                                                      out_weight);
     count_launch();
     return check_launch("neighbor_tuples_kernel");

@@ -98,7 +98,10 @@ update_kernel(const T *__restrict__ points, int64_t ld, const int32_t *__restric
         }
         if (mine) {
             match[before + __popc(ballot & ((1u << lane) - 1u))] = (int32_t)(i - base);
-            if (do_labels) atomicAdd(&hist[point_labels[i]], 1);
+            if (do_labels) {
+                const int32_t lab = point_labels[i];   // a label outside [0, num_classes) has no bin: it is not counted
+                if ((uint32_t)lab < (uint32_t)num_classes) atomicAdd(&hist[lab], 1);
+            }
         }
         if (tid == 0) n_match = all;
         __syncthreads();
