@@ -247,6 +247,34 @@ fi_status_t fi_merge_shard_lookups(int32_t shards, int32_t batch, int32_t k, con
                                    float threshold, const fi_lookup_out_t *out, void *cuda_stream);
 
 /*
+ * Dimensionality reduction in front of the look-up (Sec. 3: a one-layer network whose hidden layer has 1,024 nodes;
+ * its hidden activations are what the caches hold and what a request is looked up with).  The trained weights are
+ * the caller's; the library applies them:  y = max(0, W x + b), W [out_dim x in_dim] bf16 row-major, b [out_dim]
+ * fp32 (null: zero), products accumulated in fp32 on the tensor cores, y rounded to bf16 (nearest even).  The paper
+ * names no non-linearity; the rectifier is this library's reading.
+ *   fi_projection_create: in_dim a multiple of 8, out_dim a multiple of 16; owns a copy of the weights, its scratch
+ *     and one [max_batch x out_dim] output buffer.
+ *   fi_projection_set_weights: device pointers; copies them (asynchronous on the stream).
+ *   fi_projection_apply: x [batch_max x ld_elems] bf16 device, 16-byte aligned rows; row_idx (nullable) gathers rows of
+ *     x as in fi_cache_lookup_batch; batch_count_dev (nullable) is the device-resident row count; y [batch_max x ld_y]
+ *     bf16 device, 16-byte aligned, ld_y a multiple of 8; rows past the count are left untouched.  Asynchronous.
+ *   fi_cascade_step_projected: fi_cascade_step with the projection applied to the surviving requests' activations
+ *     first; `cache` holds projected vectors (dim = out_dim, bf16).
+ *   fi_projection_poll_status: as fi_cache_poll_status, for the projection's own kernels (synchronises).
+ * Errors: FI_ERR_INVALID_ARG for sizes, alignment, a batch above max_batch or weights never set.
+ */
+typedef struct fi_projection fi_projection_t;
+fi_status_t fi_projection_create(int32_t in_dim, int32_t out_dim, int32_t device, int32_t max_batch, fi_projection_t **out);
+fi_status_t fi_projection_destroy(fi_projection_t *proj);
+fi_status_t fi_projection_set_weights(fi_projection_t *proj, const void *weights, const float *bias, void *cuda_stream);
+fi_status_t fi_projection_poll_status(fi_projection_t *proj);
+fi_status_t fi_projection_apply(const fi_projection_t *proj, const void *x, int64_t ld_elems, const int32_t *row_idx,
+                                int32_t batch_max, const int32_t *batch_count_dev, void *y, int64_t ld_y,
+                                void *cuda_stream);
+fi_status_t fi_cascade_step_projected(const fi_cache_t *cache, const fi_projection_t *proj, const void *stage_acts,
+                                      int64_t ld_elems, const fi_cascade_state_t *state, void *cuda_stream);
+
+/*
  * Self-test of the failure path: enqueue a one-thread kernel that waits, with the given limit in SM cycles (at most
  * 2e9, about a second), on a barrier that nothing completes.  The wait runs out, the kernel sets the cache's status
  * word and returns; the next fi_cache_poll_status reports FI_ERR_TIMEOUT and the device stays usable.  Nothing

@@ -219,6 +219,45 @@ def merge_shards(shard_results: Sequence[LookupResult], shard_offsets: Sequence[
     return res
 
 
+def round_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """bfloat16 bit patterns (uint16) of float64 values, round to nearest, ties to even: the kept 16 bits are the top
+    half of the float32 pattern, so the value is first rounded to the 8-bit significand directly from float64 (no
+    double rounding through float32)."""
+    x = np.asarray(x, dtype=np.float64)
+    out = np.zeros(x.shape, np.uint16)
+    nz = np.isfinite(x) & (x != 0)
+    m, e = np.frexp(np.abs(x[nz]))                       # |x| = m * 2**e, m in [0.5, 1)
+    e_min = -126 + 1                                     # smallest normal exponent in frexp's convention
+    shift = np.maximum(e, e_min)                         # below it the spacing stays that of the smallest normals
+    q = np.abs(x[nz]) / np.ldexp(1.0, shift - 8)         # in units of the last kept bit: exact, a power-of-two scaling
+    r = np.rint(q)                                       # numpy rounds halves to even
+    val = (r * np.ldexp(1.0, shift - 8)).astype(np.float32)   # exactly representable in float32
+    bits = (val.view(np.uint32) >> 16).astype(np.uint16)
+    bits |= (np.signbit(x[nz]).astype(np.uint16) << 15)
+    out[nz] = bits
+    out[np.signbit(x) & (x == 0)] = 0x8000
+    out[np.isposinf(x)] = 0x7F80
+    out[np.isneginf(x)] = 0xFF80
+    out[np.isnan(x)] = 0x7FC0
+    return out
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    return (np.asarray(bits, dtype=np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def project(x: np.ndarray, weights: np.ndarray, bias: Optional[np.ndarray] = None):
+    """Dimensionality reduction in front of the look-up (Sec. 3): y = max(0, W x + b) per row of x, in float64 on the
+    stored values, then rounded once to bfloat16.  Returns (bf16 bit patterns [B, out], W x + b before the rectifier,
+    sum_j |w_j x_j| + |b|: the magnitude a rounding-error bound scales with)."""
+    xv = bf16_bits_to_f64(x) if x.dtype == np.uint16 else np.asarray(x, np.float64)
+    wv = bf16_bits_to_f64(weights) if weights.dtype == np.uint16 else np.asarray(weights, np.float64)
+    b = np.zeros(wv.shape[0]) if bias is None else np.asarray(bias, np.float64)
+    pre = xv @ wv.T + b
+    mag = np.abs(xv) @ np.abs(wv).T + np.abs(b)
+    return round_to_bf16_bits(np.maximum(pre, 0.0)), pre, mag
+
+
 def compact(active: np.ndarray, hit: np.ndarray) -> np.ndarray:
     """Ids of `active` whose look-up missed, order kept (Sec. 5, batch reconstruction)."""
     a = np.ascontiguousarray(active, dtype=np.int32)

@@ -15,6 +15,7 @@ import torch
 from . import build as _build
 
 FI_OK = 0
+FI_ERR_INVALID_ARG, FI_ERR_CAPACITY, FI_ERR_OOM, FI_ERR_CUDA, FI_ERR_UNSUPPORTED, FI_ERR_TIMEOUT = 1, 2, 3, 4, 5, 6
 FI_F32, FI_BF16 = 0, 1
 FI_HIT_CONF_GT, FI_HIT_DIST_LE = 0, 1
 FI_METRIC_SQL2, FI_METRIC_L2 = 0, 1
@@ -23,7 +24,9 @@ FI_PATH_AUTO, FI_PATH_STREAM, FI_PATH_GEMM = 0, 1, 2
 EXPORTS = ["fi_cache_create", "fi_cache_destroy", "fi_cache_insert", "fi_cache_set_threshold", "fi_cache_set_path",
            "fi_cache_size", "fi_cache_lookup_batch", "fi_cascade_init", "fi_cascade_step", "fi_cache_lookup_batch_host",
            "fi_cascade_run_host", "fi_cache_poll_status", "fi_cache_set_profiling",
-           "fi_cache_read_profile", "fi_lookup_noalloc", "fi_cache_compute_threshold", "fi_cache_clear", "fi_kmeans_step", "fi_cache_selftest_wait", "fi_cache_neighbor_tuples", "fi_merge_shard_lookups", "fi_launch_count", "fi_last_error", "fi_status_string"]
+           "fi_cache_read_profile", "fi_lookup_noalloc", "fi_cache_compute_threshold", "fi_cache_clear", "fi_kmeans_step", "fi_cache_selftest_wait", "fi_cache_neighbor_tuples", "fi_merge_shard_lookups",
+           "fi_projection_create", "fi_projection_destroy", "fi_projection_set_weights", "fi_projection_apply", "fi_projection_poll_status",
+           "fi_cascade_step_projected", "fi_launch_count", "fi_last_error", "fi_status_string"]
 
 
 class fi_cache_config_t(ctypes.Structure):
@@ -80,6 +83,12 @@ def load_library(path: Optional[str] = None):
     lib.fi_cache_neighbor_tuples.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp]
     lib.fi_merge_shard_lookups.argtypes = [i32, i32, i32, vp, vp, vp, vp, i32, i32, ctypes.c_float,
                                            ctypes.POINTER(fi_lookup_out_t), vp]
+    lib.fi_projection_create.argtypes = [i32, i32, i32, i32, ctypes.POINTER(vp)]
+    lib.fi_projection_destroy.argtypes = [vp]
+    lib.fi_projection_set_weights.argtypes = [vp, vp, vp, vp]
+    lib.fi_projection_poll_status.argtypes = [vp]
+    lib.fi_projection_apply.argtypes = [vp, vp, i64, vp, i32, vp, vp, i64, vp]
+    lib.fi_cascade_step_projected.argtypes = [vp, vp, vp, i64, ctypes.POINTER(fi_cascade_state_t), vp]
     lib.fi_cache_selftest_wait.argtypes = [vp, i64, vp]
     lib.fi_kmeans_step.argtypes = [vp, vp, i64, vp, i64, vp, vp, vp, vp, vp, vp]
     lib.fi_cache_compute_threshold.argtypes = [vp, vp, i64, vp, i64, ctypes.POINTER(ctypes.c_float),
@@ -314,6 +323,58 @@ def lookup_noalloc(cache_vecs: torch.Tensor, labels: torch.Tensor, weights: torc
     return out
 
 
+class Projection:
+    """The dimensionality reduction in front of the look-up (Sec. 3): y = max(0, W x + b) in bf16."""
+
+    def __init__(self, *, in_dim: int, out_dim: int = 1024, device: int = 0, max_batch: int = 1024):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p()
+        self.in_dim, self.out_dim, self.max_batch = in_dim, out_dim, max_batch
+        self.device = torch.device("cuda", device)
+        _check(self._lib.fi_projection_create(in_dim, out_dim, device, max_batch, ctypes.byref(self._h)))
+
+    # -- fi_projection_destroy
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self._lib.fi_projection_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def handle(self) -> ctypes.c_void_p:
+        return self._h
+
+    # -- fi_projection_set_weights
+    def set_weights(self, weights: torch.Tensor, bias: Optional[torch.Tensor] = None) -> None:
+        if weights.dtype != torch.bfloat16 or tuple(weights.shape) != (self.out_dim, self.in_dim) \
+                or not weights.is_contiguous() or weights.device != self.device:
+            raise ValueError("weights must be a contiguous bf16 [out_dim, in_dim] tensor on the projection's device")
+        if bias is not None and (bias.dtype != torch.float32 or bias.numel() != self.out_dim or bias.device != self.device):
+            raise ValueError("bias must be float32 [out_dim] on the projection's device")
+        _check(self._lib.fi_projection_set_weights(self._h, _dp(weights), _dp(bias), _stream_ptr(self.device)))
+
+    # -- fi_projection_poll_status
+    def poll_status(self) -> None:
+        _check(self._lib.fi_projection_poll_status(self._h))
+
+    # -- fi_projection_apply
+    def apply(self, x: torch.Tensor, row_idx: Optional[torch.Tensor] = None, count: Optional[torch.Tensor] = None,
+              out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        if x.dtype != torch.bfloat16 or x.dim() != 2 or x.shape[1] != self.in_dim or x.stride(1) != 1 or x.device != self.device:
+            raise ValueError("x must be a bf16 [batch, in_dim] tensor on the projection's device with unit inner stride")
+        batch = int(row_idx.numel()) if row_idx is not None else int(x.shape[0])
+        if out is None:
+            out = torch.zeros(batch, self.out_dim, dtype=torch.bfloat16, device=self.device)
+        _check(self._lib.fi_projection_apply(self._h, _dp(x), x.stride(0), _dp(row_idx), batch, _dp(count), _dp(out),
+                                             out.stride(0), _stream_ptr(self.device)))
+        return out
+
+
 def merge_shard_lookups(dist: torch.Tensor, global_idx: torch.Tensor, label: torch.Tensor, weight: torch.Tensor, *,
                         metric: int = FI_METRIC_SQL2, rule: int = FI_HIT_CONF_GT, threshold: float = 0.0) -> LookupOut:
     """fi_merge_shard_lookups on gathered tuples of shape [shards, batch, k]."""
@@ -366,6 +427,17 @@ def cascade_step(cache: FreezeCache, stage_acts: torch.Tensor, state: CascadeSta
     st = state.struct_for_stage(stage)
     _check(load_library().fi_cascade_step(cache.handle, _dp(stage_acts), stage_acts.stride(0), ctypes.byref(st),
                                           _stream_ptr(cache.device)))
+    state.stage = stage + 1
+
+
+def cascade_step_projected(cache: FreezeCache, proj: Projection, stage_acts: torch.Tensor, state: CascadeState,
+                           stage: Optional[int] = None) -> None:
+    """fi_cascade_step_projected: project the survivors' activations, look them up, compact the misses."""
+    if stage is None:
+        stage = state.stage
+    st = state.struct_for_stage(stage)
+    _check(load_library().fi_cascade_step_projected(cache.handle, proj.handle, _dp(stage_acts), stage_acts.stride(0),
+                                                    ctypes.byref(st), _stream_ptr(cache.device)))
     state.stage = stage + 1
 
 

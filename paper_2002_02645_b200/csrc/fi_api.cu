@@ -182,6 +182,16 @@ fi_status_t check_launch(const char *what) {
 
 using namespace fi;
 
+// The projection object behind its opaque handle: the weight rows live in a cache object of their own (its rows are
+// the B operand of the product, its per-row weights hold the bias), plus an output buffer for the cascade step.
+struct fi_projection {
+    fi_cache *w;
+    int32_t in_dim, out_dim, max_batch, device;
+    int32_t *zero_labels;   // [out_dim]
+    float *zero_bias;       // [out_dim]
+    void *y;                // [max_batch x out_dim] bf16, used by fi_cascade_step_projected
+};
+
 extern "C" {
 
 fi_status_t fi_cache_create(const fi_cache_config_t *cfg, fi_cache_t **out) {
@@ -700,6 +710,160 @@ fi_status_t fi_merge_shard_lookups(int32_t shards, int32_t batch, int32_t k, con
     }
     return launch_merge_vote(shards, batch, k, dist, global_idx, label, weight, metric, rule, threshold, *out,
                              static_cast<cudaStream_t>(cuda_stream));
+}
+
+fi_status_t fi_projection_destroy(fi_projection_t *p) {
+    if (!p) return FI_OK;
+    {
+        DeviceGuard guard(p->device);
+        cudaDeviceSynchronize();
+        cudaFree(p->zero_labels);
+        cudaFree(p->zero_bias);
+        cudaFree(p->y);
+        cudaGetLastError();
+    }
+    fi_cache_destroy(p->w);
+    delete p;
+    return FI_OK;
+}
+
+fi_status_t fi_projection_create(int32_t in_dim, int32_t out_dim, int32_t device, int32_t max_batch, fi_projection_t **out) {
+    if (out) *out = nullptr;
+    if (!out || in_dim < 8 || in_dim % 8 != 0 || out_dim < 16 || out_dim % 16 != 0 || max_batch < 1) {
+        set_error("fi_projection_create: need in_dim a multiple of 8, out_dim a multiple of 16, max_batch >= 1");
+        return FI_ERR_INVALID_ARG;
+    }
+    fi_projection *p = new (std::nothrow) fi_projection();
+    if (!p) {
+        set_error("fi_projection_create: out of host memory");
+        return FI_ERR_OOM;
+    }
+    memset(p, 0, sizeof *p);
+    p->in_dim = in_dim;
+    p->out_dim = out_dim;
+    p->max_batch = max_batch;
+    p->device = device;
+    fi_cache_config_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.dim = in_dim;
+    cfg.dtype = FI_BF16;
+    cfg.capacity = out_dim;
+    cfg.num_classes = 1;
+    cfg.k = 1;
+    cfg.rule = FI_HIT_CONF_GT;
+    cfg.metric = FI_METRIC_SQL2;
+    cfg.device = device;
+    cfg.max_batch = max_batch;
+    cfg.path = FI_PATH_GEMM;
+    fi_status_t st = fi_cache_create(&cfg, &p->w);
+    if (st != FI_OK) {
+        delete p;
+        return st;
+    }
+    DeviceGuard guard(device);
+    const size_t units = product_dump_units(max_batch, out_dim, p->w->sm_count);
+    st = dev_alloc(&p->w->tail_dump, units * 256 * 256, "allocating the projection's partial sums");
+    if (st == FI_OK) p->w->tail_dump_units = units;
+    if (st == FI_OK) st = dev_alloc(&p->zero_labels, (size_t)out_dim, "allocating the projection's labels");
+    if (st == FI_OK) st = dev_alloc(&p->zero_bias, (size_t)out_dim, "allocating the projection's zero bias");
+    unsigned char *y = nullptr;
+    if (st == FI_OK) st = dev_alloc(&y, (size_t)max_batch * out_dim * 2, "allocating the projection's output");
+    p->y = y;
+    if (st == FI_OK) {
+        cudaError_t e = cudaMemset(p->zero_labels, 0, (size_t)out_dim * sizeof(int32_t));
+        if (e == cudaSuccess) e = cudaMemset(p->zero_bias, 0, (size_t)out_dim * sizeof(float));
+        if (e != cudaSuccess) st = cuda_fail(e, "fi_projection_create: clearing buffers");
+    }
+    if (st != FI_OK) {
+        fi_projection_destroy(p);
+        return st;
+    }
+    *out = p;
+    return FI_OK;
+}
+
+fi_status_t fi_projection_set_weights(fi_projection_t *p, const void *weights, const float *bias, void *cuda_stream) {
+    if (!p || !weights) {
+        set_error("fi_projection_set_weights: null argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    fi_cache_clear(p->w);
+    return fi_cache_insert(p->w, weights, p->zero_labels, bias ? bias : p->zero_bias, p->out_dim, cuda_stream);
+}
+
+fi_status_t fi_projection_poll_status(fi_projection_t *p) {
+    if (!p) {
+        set_error("fi_projection_poll_status: null projection");
+        return FI_ERR_INVALID_ARG;
+    }
+    return fi_cache_poll_status(p->w);
+}
+
+fi_status_t fi_projection_apply(const fi_projection_t *p, const void *x, int64_t ld_elems, const int32_t *row_idx,
+                                int32_t batch_max, const int32_t *batch_count_dev, void *y, int64_t ld_y,
+                                void *cuda_stream) {
+    if (!p || batch_max < 0 || (batch_max > 0 && (!x || !y))) {
+        set_error("fi_projection_apply: null or negative argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    if (batch_max > p->max_batch || p->w->size != p->out_dim) {
+        set_error("fi_projection_apply: batch %d exceeds max_batch %d, or the weights were never set", batch_max, p->max_batch);
+        return FI_ERR_INVALID_ARG;
+    }
+    if (ld_elems < p->in_dim || ld_elems % 8 != 0 || (reinterpret_cast<uintptr_t>(x) & 15) != 0 || ld_y < p->out_dim) {
+        set_error("fi_projection_apply: rows must start on 16-byte boundaries (ld %lld, in_dim %d; ld_y %lld, out_dim %d)",
+                  (long long)ld_elems, p->in_dim, (long long)ld_y, p->out_dim);
+        return FI_ERR_INVALID_ARG;
+    }
+    if (batch_max == 0) return FI_OK;
+    DeviceGuard guard(p->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    fi_cache *w = p->w;
+    const void *src = x;
+    int64_t ld = ld_elems;
+    if (row_idx) {
+        fi_status_t st = launch_gather_rows(x, ld_elems, row_idx, batch_max, batch_count_dev, w->q_compact, p->in_dim, 2, stream);
+        if (st != FI_OK) return st;
+        src = w->q_compact;
+        ld = p->in_dim;
+    }
+    return launch_gemm_project(w, src, ld, batch_max, batch_count_dev, y, ld_y, stream);
+}
+
+fi_status_t fi_cascade_step_projected(const fi_cache_t *cache, const fi_projection_t *proj, const void *stage_acts,
+                                      int64_t ld_elems, const fi_cascade_state_t *state, void *cuda_stream) {
+    if (!cache || !proj || !state || state->batch0 < 0 || !state->miss_idx || !state->miss_count ||
+        (state->batch0 > 0 && (!stage_acts || !state->final_label || !state->exit_stage || !state->final_conf))) {
+        set_error("fi_cascade_step_projected: null or negative argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    if (cache->cfg.dtype != FI_BF16 || cache->cfg.dim != proj->out_dim || cache->cfg.device != proj->device) {
+        set_error("fi_cascade_step_projected: the cache must be bf16, of the projection's output size and on its device");
+        return FI_ERR_INVALID_ARG;
+    }
+    if (state->batch0 > cache->cfg.max_batch || state->batch0 > proj->max_batch) {
+        set_error("fi_cascade_step_projected: batch %d exceeds max_batch", state->batch0);
+        return FI_ERR_INVALID_ARG;
+    }
+    if (state->miss_idx == state->active_idx) {
+        set_error("fi_cascade_step_projected: miss_idx must not alias active_idx");
+        return FI_ERR_INVALID_ARG;
+    }
+    // slot i of the projected batch is the i-th active request: the look-up then needs no gather list
+    fi_status_t st = fi_projection_apply(proj, stage_acts, ld_elems, state->active_idx, state->batch0, state->active_count,
+                                         proj->y, proj->out_dim, cuda_stream);
+    if (st != FI_OK) return st;
+    fi_cache *c = const_cast<fi_cache *>(cache);
+    fi_lookup_out_t out;
+    out.label = c->slot_label;
+    out.conf = c->slot_conf;
+    out.hit = c->slot_hit;
+    out.topk_dist = nullptr;
+    out.topk_idx = nullptr;
+    st = fi_cache_lookup_batch(cache, proj->y, proj->out_dim, nullptr, state->batch0, state->active_count, &out, cuda_stream);
+    if (st != FI_OK) return st;
+    DeviceGuard guard(cache->cfg.device);
+    return launch_compact(c, *state, static_cast<cudaStream_t>(cuda_stream));
 }
 
 fi_status_t fi_cache_selftest_wait(fi_cache_t *c, int64_t limit_cycles, void *cuda_stream) {

@@ -235,6 +235,7 @@ struct Schedule {
     __device__ __forceinline__ int num_items() const {
         if (plan.m_tiles == 0 || n16 == 0) return 0;
         if (plan.mode == 0) return my_groups * tiles;
+        if (plan.mode == 2) return cta < plan.pieces ? (plan.pieces - cta + num_ctas - 1) / num_ctas : 0;
         return 1 + (cta < plan.tail_tiles * plan.tail_slices ? 1 : 0);
     }
     // wave + tail: the id-th tile in (cache-row tile, query tile) order; cache-row tiles are as even as 16-row
@@ -264,6 +265,16 @@ struct Schedule {
             it.emit = t == tiles - 1;
             return;
         }
+        if (plan.mode == 2) {
+            const int piece = cta + idx * num_ctas;
+            const int sl = piece % plan.tail_slices;
+            tile_of(piece / plan.tail_slices, it);
+            it.kb0 = (int)((long long)num_kb * sl / plan.tail_slices);
+            it.kb1 = (int)((long long)num_kb * (sl + 1) / plan.tail_slices);
+            it.select = it.reset = it.emit = false;
+            it.dump_slot = piece;
+            return;
+        }
         if (idx == 0) {
             tile_of(cta, it);
             it.kb0 = 0;
@@ -287,7 +298,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                    const __grid_constant__ CUtensorMap tmap_x16, const float *__restrict__ norms, long long n_entries,
                    int dim, int batch_max, const int32_t *__restrict__ count_dev, int k,
                    float *__restrict__ part_score, int32_t *__restrict__ part_idx, GemmPlan *__restrict__ plan_out,
-                   int32_t *row_bound, float *__restrict__ tail_dump, int32_t *__restrict__ status) {
+                   int32_t *row_bound, float *__restrict__ tail_dump, int32_t *__restrict__ status, int product_only) {
     constexpr int kTileRows = kTileM * MSUB;
     constexpr int kATileBytes = kABytes * MSUB;
     constexpr int kAccBufs = MSUB == 1 ? 2 : 1;   // accumulator sets in TMEM
@@ -307,7 +318,8 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     if (threadIdx.x == 0) {
         int count = count_dev ? min(*count_dev, batch_max) : batch_max;
         if (count < 0) count = 0;
-        ctl->plan = make_gemm_plan(count, n_entries, (int)gridDim.x, k, kTileRows, num_kb);
+        ctl->plan = product_only ? make_product_plan(count, n_entries, (int)gridDim.x, kTileRows, num_kb)
+                                 : make_gemm_plan(count, n_entries, (int)gridDim.x, k, kTileRows, num_kb);
         ctl->abort_flag = 0;
         if (blockIdx.x == 0) *plan_out = ctl->plan;
     }
@@ -598,6 +610,28 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             }
         };
 
+        // a piece of a tile: store the partial sums, column-major so that the 32 rows of a warp coalesce
+        auto dump_tile = [&](const WorkItem &it) {
+            const uint32_t acc = tile_no % kAccBufs, acc_ph = (tile_no / kAccBufs) & 1;
+            ++tile_no;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (acc + msub) * kMaxTileN;
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, status, 5));
+            if (!ok) return;
+            tc_fence_after();
+            float *dst = tail_dump + ((long long)it.dump_slot * kMaxTileN) * kTileRows + row_in_tile;
+            for (int c0 = first; c0 < it.w; c0 += kStep) {
+                uint32_t v[16];
+                __syncwarp();
+                tmem_ld16(taddr + c0, v);
+                tmem_ld_wait(v);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) dst[(long long)(c0 + j) * kTileRows] = __uint_as_float(v[j]);
+            }
+            tc_fence_before();
+            mbar_arrive(&ctl->tmem_empty[acc]);
+            __syncwarp();
+        };
+
         if (plan.mode == 0) {
             for (int g = 0; g < sched.my_groups && ok; ++g) {
                 const int m_tile = g * plan.mg + sched.m_local;
@@ -608,34 +642,21 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 }
                 if (ok) emit_list(m_tile, MSUB == 1 ? sched.q * 2 + half : sched.q);
             }
-        } else {
+        } else if (plan.mode == 1) {
             WorkItem it;
             sched.item(0, 0, 0, it);
             top.reset();
             select_tile(it.m_tile, it.col0, it.w);
             if (ok) emit_list(it.m_tile, it.list);
             if (ok && n_items > 1) {
-                // tail piece: store the partial sums, column-major so that the 32 rows of a warp coalesce
                 sched.item(1, 0, 0, it);
-                const uint32_t acc = tile_no % kAccBufs, acc_ph = (tile_no / kAccBufs) & 1;
-                ++tile_no;
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (acc + msub) * kMaxTileN;
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, status, 5));
-                if (ok) {
-                    tc_fence_after();
-                    float *dst = tail_dump + ((long long)it.dump_slot * kMaxTileN) * kTileRows + row_in_tile;
-                    for (int c0 = first; c0 < it.w; c0 += kStep) {
-                        uint32_t v[16];
-                        __syncwarp();
-                        tmem_ld16(taddr + c0, v);
-                        tmem_ld_wait(v);
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) dst[(long long)(c0 + j) * kTileRows] = __uint_as_float(v[j]);
-                    }
-                    tc_fence_before();
-                    mbar_arrive(&ctl->tmem_empty[acc]);
-                    __syncwarp();
-                }
+                dump_tile(it);
+            }
+        } else {
+            for (int idx = 0; idx < n_items && ok; ++idx) {
+                WorkItem it;
+                sched.item(idx, 0, 0, it);
+                dump_tile(it);
             }
         }
     }
@@ -716,6 +737,46 @@ tail_select_kernel(const GemmPlan *__restrict__ plan_dev, int num_ctas, const fl
     }
 }
 
+// Plain product, step 2: add up the pieces of every 256 x 256 tile in their order, add the bias, apply the
+// rectifier and round to bf16 (round to nearest even).  Grid (tiles, 16 column groups), one row per thread; a thread
+// writes 16 consecutive outputs of its row (32 bytes).
+__global__ void __launch_bounds__(2 * kTileM)
+product_reduce_kernel(const GemmPlan *__restrict__ plan_dev, const float *__restrict__ dump, const float *__restrict__ bias,
+                      long long n_rows, __nv_bfloat16 *__restrict__ y, long long ld_y) {
+    const GemmPlan plan = *plan_dev;
+    if (plan.mode != 2) return;
+    constexpr int kRows = 2 * kTileM;
+    const long long n16 = (n_rows + 15) / 16;
+    for (int tile = blockIdx.x; tile < plan.tail_tiles; tile += gridDim.x) {
+        const int n = tile / plan.m_tiles, m_tile = tile % plan.m_tiles;
+        const long long b0 = n16 * n / plan.n_tiles, b1 = n16 * (n + 1) / plan.n_tiles;
+        const int col0 = (int)(b0 * 16), w = (int)((b1 - b0) * 16);
+        const int c0 = blockIdx.y * 16;
+        if (c0 >= w) continue;
+        const float *base = dump + ((long long)tile * plan.tail_slices * kMaxTileN + c0) * kRows + threadIdx.x;
+        float dot[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) dot[j] = 0.f;
+        for (int sl = 0; sl < plan.tail_slices; ++sl) {
+            const float *p = base + (long long)sl * kMaxTileN * kRows;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) dot[j] += p[j * kRows];
+        }
+        const int row = m_tile * kRows + threadIdx.x;
+        if (row >= plan.count) continue;
+        __align__(16) __nv_bfloat16 out[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int c = col0 + c0 + j;
+            const float v = (long long)c < n_rows ? dot[j] + __ldg(bias + c) : 0.f;
+            out[j] = __float2bfloat16_rn(fmaxf(v, 0.f));
+        }
+        uint4 *dst = reinterpret_cast<uint4 *>(y + (long long)row * ld_y + col0 + c0);
+        dst[0] = reinterpret_cast<const uint4 *>(out)[0];
+        dst[1] = reinterpret_cast<const uint4 *>(out)[1];
+    }
+}
+
 // Exercises the bounded wait on purpose: one thread waits on a barrier that nothing will ever complete, with a
 // short limit, and must come back with the status word set instead of hanging.
 __global__ void wait_selftest_kernel(long long limit_cycles, int32_t *status) {
@@ -788,7 +849,7 @@ fi_status_t launch_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, con
     kern<<<c->sm_count, kGemmThreads, kGemmSmemBytes, stream>>>(tq, c->tmap_rows64, c->tmap_rows16, c->norms,
                                                                (long long)c->size, c->cfg.dim, batch_max, count_dev,
                                                                c->cfg.k, c->part_score, c->part_idx, c->plan_dev,
-                                                               c->row_bound, c->tail_dump, c->status_dev);
+                                                               c->row_bound, c->tail_dump, c->status_dev, 0);
     count_launch();
     fi_status_t st = check_launch("gemm_select_kernel");
     if (st != FI_OK || !tail_possible) return st;
@@ -895,6 +956,55 @@ fi_status_t launch_gemm_select(fi_cache *c, const void *queries_compact, int64_t
     }
     if (gemm_tile_m(batch_max, c->cfg.dim) == kTileM) return launch_msub<1>(c, tq, batch_max, count_dev, false, stream);
     return launch_msub<2>(c, tq, batch_max, count_dev, tail_possible, stream);
+}
+
+size_t product_dump_units(int max_batch, int64_t n_rows, int sm_count) {
+    const int m_tiles = (max_batch + 2 * kTileM - 1) / (2 * kTileM);
+    const int64_t n_tiles = ((n_rows + 15) / 16 + 15) / 16;
+    const size_t tiles = (size_t)m_tiles * (size_t)n_tiles;
+    return tiles > (size_t)sm_count ? tiles : (size_t)sm_count;   // pieces = tiles x floor(CTAs / tiles), or the tiles
+}
+
+fi_status_t launch_gemm_project(fi_cache *w, const void *queries_compact, int64_t ld_elems, int32_t batch_max,
+                                const int32_t *count_dev, void *y, int64_t ld_y, cudaStream_t stream) {
+    if (batch_max <= 0) return FI_OK;
+    fi_status_t st = ensure_tensor_maps(w);
+    if (st != FI_OK) return st;
+    if ((reinterpret_cast<uintptr_t>(queries_compact) & 15) != 0 || (ld_elems % 8) != 0 ||
+        (reinterpret_cast<uintptr_t>(y) & 15) != 0 || (ld_y % 8) != 0 || (w->size % 16) != 0) {
+        set_error("projection: inputs and outputs must be 16-byte aligned, leading dimensions multiples of 8, outputs a multiple of 16");
+        return FI_ERR_INVALID_ARG;
+    }
+    if (w->tail_dump_units < product_dump_units(batch_max, w->size, w->sm_count)) {
+        set_error("projection: partial-sum buffer too small for a batch of %d", batch_max);
+        return FI_ERR_INVALID_ARG;
+    }
+    CUtensorMap tq;
+    st = encode_bf16_map(&tq, queries_compact, (uint64_t)batch_max, (uint64_t)w->cfg.dim, (uint64_t)ld_elems, kTileM);
+    if (st != FI_OK) return st;
+    static bool attr_set = false;
+    auto kern = gemm_select_kernel<8, 2>;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) != cudaSuccess) {
+            set_error("cannot reserve %d bytes of shared memory for the projection", kGemmSmemBytes);
+            cudaGetLastError();
+            return FI_ERR_CUDA;
+        }
+        attr_set = true;
+    }
+    kern<<<w->sm_count, kGemmThreads, kGemmSmemBytes, stream>>>(tq, w->tmap_rows64, w->tmap_rows16, w->norms,
+                                                               (long long)w->size, w->cfg.dim, batch_max, count_dev, 1,
+                                                               w->part_score, w->part_idx, w->plan_dev, w->row_bound,
+                                                               w->tail_dump, w->status_dev, 1);
+    count_launch();
+    st = check_launch("gemm_select_kernel (product)");
+    if (st != FI_OK) return st;
+    const int m_tiles = (batch_max + 2 * kTileM - 1) / (2 * kTileM);
+    const int n_tiles = (int)(((w->size + 15) / 16 + 15) / 16);
+    product_reduce_kernel<<<dim3(m_tiles * n_tiles, kMaxTileN / 16), 2 * kTileM, 0, stream>>>(
+        w->plan_dev, w->tail_dump, w->weights, (long long)w->size, static_cast<__nv_bfloat16 *>(y), (long long)ld_y);
+    count_launch();
+    return check_launch("product_reduce_kernel");
 }
 
 }  // namespace fi

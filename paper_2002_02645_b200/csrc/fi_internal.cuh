@@ -42,11 +42,11 @@ struct GemmPlan {
     int32_t list_len;     // entries per candidate list
     int32_t tile_m;       // query rows per CTA tile
     int32_t lists;        // candidate lists per query
-    int32_t mode;         // 0 = ranges, 1 = wave + tail
-    int32_t n_tiles;      // wave + tail: cache-row tiles per query tile
-    int32_t tail_tiles;   // wave + tail: tiles beyond the first wave
-    int32_t tail_slices;  // wave + tail: pieces each of those is cut into along the row length
-    int32_t pad;
+    int32_t mode;         // 0 = ranges, 1 = wave + tail, 2 = pieces only (plain product, no select)
+    int32_t n_tiles;      // wave + tail, pieces: cache-row tiles per query tile
+    int32_t tail_tiles;   // wave + tail: tiles beyond the first wave; pieces: all tiles
+    int32_t tail_slices;  // wave + tail, pieces: pieces each of those tiles is cut into along the row length
+    int32_t pieces;       // pieces: tail_tiles * tail_slices
 };
 
 __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entries, int num_ctas, int k, int tile_m,
@@ -56,7 +56,7 @@ __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entrie
     p.m_tiles = (count + tile_m - 1) / tile_m;
     p.list_len = gemm_list_len(k);
     p.tile_m = tile_m;
-    p.pad = 0;
+    p.pieces = 0;
     p.lists = 0;
     p.mode = 0;
     p.n_tiles = p.tail_tiles = p.tail_slices = 0;
@@ -115,9 +115,31 @@ __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entrie
     return p;
 }
 
-struct LaunchCtx {
-    cudaStream_t stream;
-};
+// Plan of a plain product Y = Q W^T (the projection in front of the look-up): every 256 x 256 tile of Y is cut
+// along the row length into as many pieces as fill the CTAs once; piece p = tile * slices + slice goes to CTA
+// p mod num_ctas and leaves its partial sums in slot p.
+__host__ __device__ inline GemmPlan make_product_plan(int count, long long n_rows, int num_ctas, int tile_m, int num_kb) {
+    GemmPlan p;
+    p.count = count;
+    p.m_tiles = (count + tile_m - 1) / tile_m;
+    p.mg = p.m_tiles > 0 ? p.m_tiles : 1;
+    p.groups = 1;
+    p.range16 = 16;
+    p.list_len = 0;
+    p.tile_m = tile_m;
+    p.lists = 0;
+    p.mode = 2;
+    const long long n16 = (n_rows + 15) / 16;
+    p.n_tiles = (int32_t)((n16 + 15) / 16);
+    p.parts = p.n_tiles;
+    p.tail_tiles = p.m_tiles * p.n_tiles;
+    int slices = p.tail_tiles > 0 ? num_ctas / p.tail_tiles : 1;
+    if (slices > num_kb) slices = num_kb;
+    if (slices < 1) slices = 1;
+    p.tail_slices = slices;
+    p.pieces = p.tail_tiles * slices;
+    return p;
+}
 
 }  // namespace fi
 
@@ -214,6 +236,11 @@ fi_status_t launch_neighbor_tuples(const fi_cache *c, const int32_t *topk_idx, i
 fi_status_t launch_merge_vote(int shards, int batch, int k, const float *dist, const int32_t *idx, const int32_t *label,
                               const float *weight, int metric, int rule, float tau, const fi_lookup_out_t &out,
                               cudaStream_t stream);
+// plain product on the tensor cores: y = max(0, q W^T + bias) rounded to bf16, W = the rows held in `w`, bias = its
+// per-row weights; `units` = slots of partial sums `w->tail_dump` must hold (see product_dump_units)
+fi_status_t launch_gemm_project(fi_cache *w, const void *queries_compact, int64_t ld_elems, int32_t batch_max,
+                                const int32_t *count_dev, void *y, int64_t ld_y, cudaStream_t stream);
+size_t product_dump_units(int max_batch, int64_t n_rows, int sm_count);
 fi_status_t launch_wait_selftest(fi_cache *c, long long limit_cycles, cudaStream_t stream);
 fi_status_t ensure_tensor_maps(fi_cache *c);
 size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, int dim);

@@ -34,6 +34,7 @@ import numpy as np
 # stream ids: one namespace per kind of draw so that no two draws share a key
 _S_MEANS, _S_CACHE_LABELS, _S_CACHE_NOISE = 1, 2, 3
 _S_QUERY_LABELS, _S_QUERY_NOISE, _S_COPIES, _S_SHUFFLE = 4, 5, 6, 7
+_S_PROJ_W, _S_PROJ_B = 8, 9
 
 _CHUNK_ELEMS = 1 << 22
 
@@ -121,6 +122,19 @@ def _fill_rows(out: np.ndarray, labels: np.ndarray, means: np.ndarray, *, kind: 
     else:
         with ThreadPoolExecutor(_workers()) as ex:
             list(ex.map(work, chunks))
+
+
+def projection_weights(in_dim: int, out_dim: int, seed: int, stage: int = 0):
+    """Random stand-in for a layer's trained dimensionality-reduction weights (the trained ones are not available):
+    W [out_dim, in_dim] ~ N(0, 1/in_dim) as bf16 bit patterns, bias [out_dim] ~ 0.1 N(0, 1) as float32."""
+    w = np.empty((out_dim, in_dim), dtype=np.uint16)
+    rows_per_chunk = max(1, _CHUNK_ELEMS // in_dim)
+    scale = np.float32(1.0 / np.sqrt(in_dim))
+    for c, lo in enumerate(range(0, out_dim, rows_per_chunk)):
+        hi = min(out_dim, lo + rows_per_chunk)
+        w[lo:hi] = f32_to_bf16_bits(_rng(seed, _S_PROJ_W, stage, c).standard_normal((hi - lo, in_dim), dtype=np.float32) * scale)
+    bias = (_rng(seed, _S_PROJ_B, stage).standard_normal(out_dim, dtype=np.float32) * np.float32(0.1)).astype(np.float32)
+    return w, bias
 
 
 def _alloc(n: int, dim: int, dtype: str) -> np.ndarray:

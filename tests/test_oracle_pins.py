@@ -452,3 +452,44 @@ def test_merge_of_row_shards_equals_the_unsharded_lookup():
     np.testing.assert_array_equal(merged.label, whole.label)
     np.testing.assert_array_equal(merged.conf, whole.conf)
     np.testing.assert_array_equal(merged.hit, whole.hit)
+
+
+# ------------------------------------------------------------------ projection in front of the look-up (Sec. 3)
+
+def test_bf16_rounding_against_the_library_conversion_and_hand_ties():
+    import torch
+    rng = np.random.default_rng(5)
+    x32 = (rng.standard_normal(100000) * 10.0 ** rng.uniform(-40, 38, 100000)).astype(np.float32)
+    x32 = np.concatenate([x32, np.array([0.0, -0.0, 1e-45, 1e-40, 3.38e38, 3.4e38, np.inf, -np.inf], np.float32)])
+    want = torch.from_numpy(x32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(fo.round_to_bf16_bits(x32.astype(np.float64)), want)   # float32 inputs: one rounding
+    # ties by hand: bf16 keeps 8 significand bits, so 1 + 2^-8 lies half-way between 1 and 1 + 2^-7
+    one, step = 0x3F80, 2.0 ** -7
+    assert fo.round_to_bf16_bits(np.array([1 + step / 2]))[0] == one            # tie -> even (1.0)
+    assert fo.round_to_bf16_bits(np.array([1 + 3 * step / 2]))[0] == one + 2    # tie -> even (1 + 2 steps)
+    assert fo.round_to_bf16_bits(np.array([1 + step / 2 + 1e-12]))[0] == one + 1
+    # a float64 value just above a tie must round up even though float32 would first land on the tie
+    assert fo.round_to_bf16_bits(np.array([1 + step / 2 + 2.0 ** -40]))[0] == one + 1
+    np.testing.assert_array_equal(fo.bf16_bits_to_f64(np.array([one, one + 1], np.uint16)), [1.0, 1 + step])
+
+
+def test_projection_hand_case_identity_and_bias():
+    w = np.array([[1.0, 2.0, -1.0, 0.0], [0.5, 0.0, 0.0, 4.0]], np.float32)
+    x = np.array([[0.5, 0.25, 3.0, 1.0], [2.0, 1.0, 0.0, -1.0]], np.float32)
+    b = np.array([0.125, -1.0], np.float32)
+    bits, pre, mag = fo.project(x, w, b)
+    np.testing.assert_array_equal(pre, [[-1.875, 3.25], [4.125, -4.0]])          # by hand
+    np.testing.assert_array_equal(mag, [[4.125, 5.25], [4.125, 6.0]])
+    np.testing.assert_array_equal(fo.bf16_bits_to_f64(bits), [[0.0, 3.25], [4.125, 0.0]])
+    # identity weights: the projection is the rectifier; bf16 inputs come back bit for bit
+    rng = np.random.default_rng(6)
+    xb = fo.round_to_bf16_bits(rng.standard_normal((5, 16)))
+    eye = fo.round_to_bf16_bits(np.eye(16))
+    got, _, _ = fo.project(xb, eye)
+    want = np.where(fo.bf16_bits_to_f64(xb) > 0, xb, 0).astype(np.uint16)
+    np.testing.assert_array_equal(got, want)
+    # operands are not transposed: a non-square W [out=3, in=16] gives 3 outputs per row
+    w3 = fo.round_to_bf16_bits(rng.standard_normal((3, 16)))
+    got3, pre3, _ = fo.project(xb, w3)
+    assert got3.shape == (5, 3)
+    np.testing.assert_allclose(pre3[2, 1], float(fo.bf16_bits_to_f64(xb[2]) @ fo.bf16_bits_to_f64(w3[1])), rtol=1e-15)
