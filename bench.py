@@ -638,6 +638,124 @@ def run_tau_sweep(args):
         c.close()
 
 
+def run_projected(args):
+    """The 4-stage cascade as the paper runs it (Sec. 3): every layer's activation is first reduced to 1,024 dimensions
+    by that layer's one-layer network, and the caches hold reduced vectors.  Random weights stand in for the trained
+    ones.  A step = cascade_init + 4 x (projection of the survivors + look-up + compaction)."""
+    import torch
+    from paper_2002_02645_b200 import binding as fb
+    from paper_2002_02645_b200 import build as fbuild
+    from paper_2002_02645_b200 import datagen as dg
+    fbuild.build_library()
+    dev = torch.device("cuda", 0)
+    out_dim = 1024
+    w = build_workload("cfg2", seed=0)
+    b0, n_stage = w.stages[0].queries.shape[0], len(w.stages)
+    projs, caches, acts, taus = [], [], [], []
+    for l, st in enumerate(w.stages):
+        w_bits, bias = dg.projection_weights(st.dim, out_dim, seed=0, stage=l)
+        p = fb.Projection(in_dim=st.dim, out_dim=out_dim, max_batch=b0)
+        p.set_weights(to_dev(w_bits, dev), torch.from_numpy(bias).to(dev))
+        c = fb.FreezeCache(dim=out_dim, capacity=st.cache_vecs.shape[0], num_classes=w.num_classes, k=w.k,
+                           dtype=fb.FI_BF16, max_batch=max(b0, st.calib.shape[0]))
+        for lo in range(0, st.cache_vecs.shape[0], b0):
+            hi = min(st.cache_vecs.shape[0], lo + b0)
+            c.insert(p.apply(to_dev(st.cache_vecs[lo:hi], dev)), torch.from_numpy(st.cache_labels[lo:hi]).to(dev))
+        taus.append(calibrate(c, p.apply(to_dev(st.calib, dev)), w.meta["percentiles"][l]))
+        projs.append(p)
+        caches.append(c)
+        acts.append(to_dev(st.queries, dev))
+    state = fb.CascadeState(b0, dev)
+
+    def step():
+        fb.cascade_init(state, n_stage)
+        for l in range(n_stage):
+            fb.cascade_step_projected(caches[l], projs[l], acts[l], state, l)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    arrivals = [b0]
+    fb.cascade_init(state, n_stage)
+    for l in range(n_stage):
+        fb.cascade_step_projected(caches[l], projs[l], acts[l], state, l)
+        arrivals.append(int(state.survivors(l)[1].item()))
+    for o in projs + caches:
+        o.set_profiling(True)
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.25)
+    l0 = fb.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    launches = fb.launch_count() - l0
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    prof_p = [p.read_profile() for p in projs]
+    prof_c = [c.read_profile() for c in caches]
+    for o in projs + caches:
+        o.set_profiling(False)
+        o.poll_status()
+
+    # end to end: host activations in pinned memory, copied in every step; results read back every step
+    host_acts = [to_pinned(st.queries) for st in w.stages]
+    dev_acts = [torch.empty_like(a) for a in acts]
+    h_label = torch.empty(b0, dtype=torch.int32).pin_memory()
+    h_stage = torch.empty(b0, dtype=torch.int32).pin_memory()
+
+    def e2e_step():
+        for d, h in zip(dev_acts, host_acts):
+            d.copy_(h, non_blocking=True)
+        fb.cascade_init(state, n_stage)
+        for l in range(n_stage):
+            fb.cascade_step_projected(caches[l], projs[l], dev_acts[l], state, l)
+        h_label.copy_(state.final_label[:b0], non_blocking=True)
+        h_stage.copy_(state.exit_stage[:b0], non_blocking=True)
+        torch.cuda.synchronize()
+
+    for _ in range(2):
+        e2e_step()
+    n_e2e = max(3, min(args.steps, 10))
+    t0 = time.perf_counter()
+    for _ in range(n_e2e):
+        e2e_step()
+    e2e_s = time.perf_counter() - t0
+    h2d = sum(int(a.numel() * a.element_size()) for a in host_acts)
+
+    peaks, src = load_peaks()
+    d0 = w.stages[0].dim
+    flops = 2.0 * b0 * out_dim * d0
+    avg_s = prof_p[0][0] / max(1, prof_p[0][1]) * 1e-3
+    achieved = flops / avg_s / 1e12
+    print(json.dumps({
+        "metric": METRIC, "value": b0 / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name + "_projected_to_1024", "stages": n_stage, "batch": b0, "k": w.k,
+                   "cache_entries": int(w.stages[0].cache_vecs.shape[0]), "dims": [s.dim for s in w.stages],
+                   "reduced_dim": out_dim, "thresholds": taus, "arrivals": arrivals,
+                   "l2": "inputs larger than L2 (activations and weights %.2f GB per step)"
+                         % (sum(2.0 * s.dim * (b0 + out_dim) for s in w.stages) / 1e9)},
+        "e2e": {"value": b0 * n_e2e / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": b0 * 8,
+                "steps": n_e2e, "ms_per_step": 1e3 * e2e_s / n_e2e},
+        "gpu_launches": int(launches), "clocks": clocks,
+        "roofline": {"bound": "tensor", "kernel": "gemm_select_kernel in product mode + product_reduce_kernel (stage 0)",
+                     "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": achieved / peaks["bf16_tflops"], "peak_source": f"cuBLAS bf16 burst, {src}",
+                     "frac_of_nominal": achieved / 2250.0, "traffic": None, "avg_launch_ms": avg_s * 1e3,
+                     "algorithmic_flops": flops, "algorithmic_bytes": 2.0 * d0 * (b0 + out_dim) + 2.0 * b0 * out_dim},
+        "stages": [{"stage": l, "arrivals": arrivals[l], "projection_ms": prof_p[l][0] / max(1, prof_p[l][1]),
+                    "distance_kernel_ms": prof_c[l][0] / max(1, prof_c[l][1])} for l in range(n_stage)],
+        "cpu_baseline": None}))
+    for o in projs + caches:
+        o.close()
+
+
 def run_rowshard(args):
     """The 200,000-entry single-layer workload with the cache ROWS split over the ranks (strong scaling: the same
     8,192 requests and the same entries at every N).  Every rank looks all requests up in its rows, one all-gather
@@ -728,7 +846,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0", "kmeans", "cfg3-rows", "tau-sweep"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0", "kmeans", "cfg3-rows", "tau-sweep", "cfg2-proj"])
     ap.add_argument("--cpu-sample", type=int, default=0,
                     help="requests per oracle timing (0: sized for 10-30 s of CPU work)")
     ap.add_argument("--batch", type=int, default=16, help="batch of the latency workload (cfg5): 1, 4 or 16")
@@ -737,6 +855,8 @@ def main():
     args = ap.parse_args()
     if args.workload == "kmeans":
         run_kmeans(args)
+    elif args.workload == "cfg2-proj" and args.impl == "ours":
+        run_projected(args)
     elif args.workload == "tau-sweep":
         run_tau_sweep(args)
     elif args.workload == "cfg3-rows" and args.impl == "ours":

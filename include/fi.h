@@ -268,6 +268,9 @@ fi_status_t fi_projection_create(int32_t in_dim, int32_t out_dim, int32_t device
 fi_status_t fi_projection_destroy(fi_projection_t *proj);
 fi_status_t fi_projection_set_weights(fi_projection_t *proj, const void *weights, const float *bias, void *cuda_stream);
 fi_status_t fi_projection_poll_status(fi_projection_t *proj);
+/* as fi_cache_set_profiling / fi_cache_read_profile, around the two kernels of fi_projection_apply */
+fi_status_t fi_projection_set_profiling(fi_projection_t *proj, int32_t enable);
+fi_status_t fi_projection_read_profile(fi_projection_t *proj, float *total_ms, int32_t *launches);
 fi_status_t fi_projection_apply(const fi_projection_t *proj, const void *x, int64_t ld_elems, const int32_t *row_idx,
                                 int32_t batch_max, const int32_t *batch_count_dev, void *y, int64_t ld_y,
                                 void *cuda_stream);

@@ -25,7 +25,8 @@ EXPORTS = ["fi_cache_create", "fi_cache_destroy", "fi_cache_insert", "fi_cache_s
            "fi_cache_size", "fi_cache_lookup_batch", "fi_cascade_init", "fi_cascade_step", "fi_cache_lookup_batch_host",
            "fi_cascade_run_host", "fi_cache_poll_status", "fi_cache_set_profiling",
            "fi_cache_read_profile", "fi_lookup_noalloc", "fi_cache_compute_threshold", "fi_cache_clear", "fi_kmeans_step", "fi_cache_selftest_wait", "fi_cache_neighbor_tuples", "fi_merge_shard_lookups",
-           "fi_projection_create", "fi_projection_destroy", "fi_projection_set_weights", "fi_projection_apply", "fi_projection_poll_status",
+           "fi_projection_create", "fi_projection_destroy", "fi_projection_set_weights", "fi_projection_apply", "fi_projection_poll_status", "fi_projection_set_profiling",
+           "fi_projection_read_profile",
            "fi_cascade_step_projected", "fi_launch_count", "fi_last_error", "fi_status_string"]
 
 
@@ -87,6 +88,8 @@ def load_library(path: Optional[str] = None):
     lib.fi_projection_destroy.argtypes = [vp]
     lib.fi_projection_set_weights.argtypes = [vp, vp, vp, vp]
     lib.fi_projection_poll_status.argtypes = [vp]
+    lib.fi_projection_set_profiling.argtypes = [vp, i32]
+    lib.fi_projection_read_profile.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.fi_projection_apply.argtypes = [vp, vp, i64, vp, i32, vp, vp, i64, vp]
     lib.fi_cascade_step_projected.argtypes = [vp, vp, vp, i64, ctypes.POINTER(fi_cascade_state_t), vp]
     lib.fi_cache_selftest_wait.argtypes = [vp, i64, vp]
@@ -361,6 +364,15 @@ class Projection:
     # -- fi_projection_poll_status
     def poll_status(self) -> None:
         _check(self._lib.fi_projection_poll_status(self._h))
+
+    # -- fi_projection_set_profiling / fi_projection_read_profile
+    def set_profiling(self, enable: bool) -> None:
+        _check(self._lib.fi_projection_set_profiling(self._h, 1 if enable else 0))
+
+    def read_profile(self):
+        ms, n = ctypes.c_float(0.0), ctypes.c_int32(0)
+        _check(self._lib.fi_projection_read_profile(self._h, ctypes.byref(ms), ctypes.byref(n)))
+        return float(ms.value), int(n.value)
 
     # -- fi_projection_apply
     def apply(self, x: torch.Tensor, row_idx: Optional[torch.Tensor] = None, count: Optional[torch.Tensor] = None,

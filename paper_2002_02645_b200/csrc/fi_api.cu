@@ -827,7 +827,26 @@ fi_status_t fi_projection_apply(const fi_projection_t *p, const void *x, int64_t
         src = w->q_compact;
         ld = p->in_dim;
     }
-    return launch_gemm_project(w, src, ld, batch_max, batch_count_dev, y, ld_y, stream);
+    prof_mark(w, 0, stream);
+    fi_status_t st = launch_gemm_project(w, src, ld, batch_max, batch_count_dev, y, ld_y, stream);
+    if (st == FI_OK) prof_mark(w, 1, stream);
+    return st;
+}
+
+fi_status_t fi_projection_set_profiling(fi_projection_t *p, int32_t enable) {
+    if (!p) {
+        set_error("fi_projection_set_profiling: null projection");
+        return FI_ERR_INVALID_ARG;
+    }
+    return fi_cache_set_profiling(p->w, enable);
+}
+
+fi_status_t fi_projection_read_profile(fi_projection_t *p, float *total_ms, int32_t *launches) {
+    if (!p) {
+        set_error("fi_projection_read_profile: null projection");
+        return FI_ERR_INVALID_ARG;
+    }
+    return fi_cache_read_profile(p->w, total_ms, launches);
 }
 
 fi_status_t fi_cascade_step_projected(const fi_cache_t *cache, const fi_projection_t *proj, const void *stage_acts,

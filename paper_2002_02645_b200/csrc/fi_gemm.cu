@@ -553,14 +553,31 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     }
                 }
                 if (__any_sync(0xFFFFFFFFu, cnt > kQueueCap)) {
-                    // a queue overflowed inside this chunk: insert what was queued before it, then this chunk
-                    // column by column (arrival order, hence the tie order, is kept)
+                    // a queue overflowed inside this chunk: insert what was queued before it (all lanes together),
+                    // then queue this chunk again against the tighter threshold; only if that overflows too (lists
+                    // still filling up) is it inserted column by column.  Arrival order, hence the tie order, is kept.
                     flush(cnt0);
-#pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        if (sc[j] < top.s[KP - 1] && sc[j] <= bound) top.insert(sc[j], col0 + c0 + j);
-                    cnt = 0;
                     thr = fminf(top.s[KP - 1], bound);
+                    cnt = 0;
+                    if (mn <= thr) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            if (sc[j] <= thr) {
+                                if (cnt < kQueueCap) {
+                                    qs[cnt * kEpiThreads] = sc[j];
+                                    qi[cnt * kEpiThreads] = col0 + c0 + j;
+                                }
+                                ++cnt;
+                            }
+                        }
+                    }
+                    if (__any_sync(0xFFFFFFFFu, cnt > kQueueCap)) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (sc[j] < top.s[KP - 1] && sc[j] <= bound) top.insert(sc[j], col0 + c0 + j);
+                        cnt = 0;
+                        thr = fminf(top.s[KP - 1], bound);
+                    }
                 }
             };
 

@@ -133,8 +133,9 @@ __host__ __device__ inline GemmPlan make_product_plan(int count, long long n_row
     p.n_tiles = (int32_t)((n16 + 15) / 16);
     p.parts = p.n_tiles;
     p.tail_tiles = p.m_tiles * p.n_tiles;
+    // a piece shorter than 8 k-blocks costs more to store and add up again than its MMAs take
     int slices = p.tail_tiles > 0 ? num_ctas / p.tail_tiles : 1;
-    if (slices > num_kb) slices = num_kb;
+    if (slices > num_kb / 8) slices = num_kb / 8;
     if (slices < 1) slices = 1;
     p.tail_slices = slices;
     p.pieces = p.tail_tiles * slices;
