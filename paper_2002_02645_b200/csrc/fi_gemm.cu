@@ -174,21 +174,20 @@ struct TopList {
             i[e] = -1;
         }
     }
-    // precondition: sc < s[KP-1].  Equal scores keep their arrival order (smaller index first).
+    // Equal scores keep their arrival order (smaller index first).  All comparisons are taken against the old
+    // list first, so the selects of the KP positions do not depend on one another (a bubble pass would chain
+    // them, and the two epilogue warps per scheduler cannot hide that latency).
     __device__ __forceinline__ void insert(float sc, int32_t idx) {
-        s[KP - 1] = sc;
-        i[KP - 1] = idx;
+        bool below[KP];
+#pragma unroll
+        for (int e = 0; e < KP; ++e) below[e] = sc < s[e];
 #pragma unroll
         for (int e = KP - 1; e > 0; --e) {
-            if (s[e] < s[e - 1]) {
-                float ts = s[e];
-                s[e] = s[e - 1];
-                s[e - 1] = ts;
-                int32_t ti = i[e];
-                i[e] = i[e - 1];
-                i[e - 1] = ti;
-            }
+            s[e] = below[e] ? (below[e - 1] ? s[e - 1] : sc) : s[e];
+            i[e] = below[e] ? (below[e - 1] ? i[e - 1] : idx) : i[e];
         }
+        s[0] = below[0] ? sc : s[0];
+        i[0] = below[0] ? idx : i[0];
     }
 };
 

@@ -85,29 +85,37 @@ __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entrie
             return p;
         }
     }
-    // pick the group size that needs the fewest MMA columns per CTA in total
+    // Group size: the fewest MMA columns per CTA in total, except that on long ranges a larger group within 3 % of
+    // that minimum is preferred: it means fewer, longer ranges, hence fewer candidate lists per query to warm up
+    // and to merge, and more CTAs streaming the same cache rows at the same time.
+    // (32-bit divisions: one thread of every CTA evaluates this at kernel start, and 64-bit ones cost microseconds)
     int best_mg = 1;
-    long long best_cost = -1;
     int mg_max = p.m_tiles < 16 ? p.m_tiles : 16;
     if (mg_max > num_ctas) mg_max = num_ctas;
+    const int n16i = (int)n16;   // entries are indexed with int32, so n16 < 2^27
+    long long cost[16], min_cost = -1;
+    int eff[16];
     for (int mg = 1; mg <= mg_max; ++mg) {
-        int groups = (p.m_tiles + mg - 1) / mg;
-        int mg_eff = (p.m_tiles + groups - 1) / groups;
-        long long parts = num_ctas / mg_eff;
-        if (parts > n16) parts = n16;
-        long long r16 = (n16 + parts - 1) / parts;
-        long long cost = (long long)groups * r16;
-        if (best_cost < 0 || cost < best_cost || (cost == best_cost && mg_eff > best_mg)) {
-            best_cost = cost;
-            best_mg = mg_eff;
-        }
+        const int groups = (p.m_tiles + mg - 1) / mg;
+        const int mg_eff = (p.m_tiles + groups - 1) / groups;
+        int cand_parts = num_ctas / mg_eff;
+        if (cand_parts > n16i) cand_parts = n16i;
+        const int r = (n16i + cand_parts - 1) / cand_parts;
+        cost[mg - 1] = (long long)groups * r;
+        eff[mg - 1] = mg_eff;
+        if (min_cost < 0 || cost[mg - 1] < min_cost) min_cost = cost[mg - 1];
+    }
+    for (int mg = 1; mg <= mg_max; ++mg) {
+        const long long c = cost[mg - 1];
+        // short ranges (under 4,096 rows per CTA) are latency-bound: exact minimum only
+        if ((min_cost >= 256 ? c * 100 <= min_cost * 103 : c == min_cost) && eff[mg - 1] > best_mg) best_mg = eff[mg - 1];
     }
     p.mg = best_mg;
     p.groups = (p.m_tiles + p.mg - 1) / p.mg;
-    long long parts = num_ctas / p.mg;
-    if (parts > n16) parts = n16;
-    long long r16 = (n16 + parts - 1) / parts;
-    parts = (n16 + r16 - 1) / r16;   // drop ranges that would be empty
+    int parts = num_ctas / p.mg;
+    if (parts > n16i) parts = n16i;
+    const int r16 = (n16i + parts - 1) / parts;
+    parts = (n16i + r16 - 1) / r16;   // drop ranges that would be empty
     p.parts = (int32_t)parts;
     p.range16 = (int32_t)r16;
     // with 128-row tiles two epilogue warps share each row and keep a list each
