@@ -269,7 +269,8 @@ fi_status_t fi_cache_create(const fi_cache_config_t *cfg, fi_cache_t **out) {
     if (st == FI_OK) need(dev_alloc(&c->slot_conf, (size_t)cfg->max_batch, "allocating slot confidences"));
     if (st == FI_OK) need(dev_alloc(&c->slot_hit, (size_t)cfg->max_batch, "allocating slot hit flags"));
     if (st == FI_OK) need(dev_alloc(&c->plan_dev, 1, "allocating the plan"));
-    if (st == FI_OK && bf16) need(dev_alloc(&c->row_bound, (size_t)cfg->max_batch + 256, "allocating the row bounds"));
+    if (st == FI_OK && bf16)
+        need(dev_alloc(&c->row_bound, ((size_t)cfg->max_batch + 256) * gemm_list_len(cfg->k), "allocating the row bounds"));
     if (st == FI_OK) need(dev_alloc(&c->status_dev, 1, "allocating the status word"));
     if (st == FI_OK) {
         cudaError_t e = cudaMemset(c->status_dev, 0, sizeof(int32_t));

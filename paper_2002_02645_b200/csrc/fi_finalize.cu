@@ -111,7 +111,7 @@ __global__ void __launch_bounds__(kFinThreads) finalize_kernel(FinalizeParams p)
         for (int e = tid; e < entries; e += kFinThreads) {
             float s = ps[e];
             int i = pi[e];
-            if (i < 0) continue;
+            if (i < 0 || i >= p.n_entries) continue;   // empty slot (an index past the cache cannot occur; never follow one)
             bool above = r == 0 || pair_less(prev_s, prev_i, s, i);
             if (above && pair_less(s, i, best_s, best_i)) {
                 best_s = s;

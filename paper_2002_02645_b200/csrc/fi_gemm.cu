@@ -301,6 +301,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     constexpr int kTileRows = kTileM * MSUB;
     constexpr int kATileBytes = kABytes * MSUB;
     constexpr int kAccBufs = MSUB == 1 ? 2 : 1;   // accumulator sets in TMEM
+    constexpr int kSlots = KP;                    // bound slots per query row
 
     extern __shared__ unsigned char smem_raw[];
     // operand stages need 1024-byte alignment for the 128-byte swizzle
@@ -481,10 +482,17 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         TopList<KP> top;
         bool ok = true;
 
-        // Bound shared by every CTA that scans cache rows for the same query: each list publishes its list_len-th
-        // best score, the minimum over lists bounds the list_len-th best of the whole cache from above, and a
-        // score above it can be skipped by every list.  Scores equal to the bound are kept, so which candidates
-        // reach the final merge never depends on the order in which CTAs publish.
+        // Bound shared by every CTA that scans cache rows for the same query.  A row has KP slots.
+        // Ranges of 4 tiles or more (sharing 2): list l lowers slot (l + e) mod KP to its e-th best score.  The KP
+        // slot values then belong to KP different cache rows (two slots filled by the same list hold different
+        // entries of it; a stale entry is only larger than the current one), so their maximum bounds the KP-th
+        // best score of the whole cache from above.  With many lists per query this is far tighter than any one
+        // list's own KP-th best.
+        // Ranges of 2 or 3 tiles (sharing 1): too short to pay for KP atomics per list; every list lowers slot 0 to
+        // its KP-th best score, which is such a bound too.  Single tiles (sharing 0): nothing to share.
+        // A score above the bound can be skipped by every list.  Scores equal to the bound are kept, so which
+        // candidates reach the final merge never depends on the order in which CTAs publish.
+        const int sharing = plan.mode != 0 || sched.tiles < 2 ? 0 : sched.tiles < 4 ? 1 : 2;
         float bound = __int_as_float(0x7F800000);
 
         // insert the first n queued candidates of every lane, all lanes together
@@ -501,14 +509,28 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         uint32_t tile_no = 0;
 
         // scan one accumulator tile into the running list of this thread's row
-        auto select_tile = [&](int m_tile, int col0, int w) {
+        auto select_tile = [&](int m_tile, int col0, int w, int list, int sharing) {
             const uint32_t acc = tile_no % kAccBufs, acc_ph = (tile_no / kAccBufs) & 1;
             ++tile_no;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (acc + msub) * kMaxTileN;
-            int32_t *my_bound = row_bound + m_tile * kTileRows + row_in_tile;
+            int32_t *my_bound = row_bound + (long long)(m_tile * kTileRows + row_in_tile) * kSlots;
             float *nrm = my_norm + acc * (kMaxTileN / 2);   // acc is 0 for 256-row tiles
-            int32_t bound_key;   // read past L1: other SMs lower it
-            asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(bound_key) : "l"(my_bound) : "memory");
+            // the row's slots, read past L1 (other SMs lower them); the bound is the largest of them
+            int32_t bound_key = 0x7F7F7F7F;
+            if (sharing == 1) {
+                asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(bound_key) : "l"(my_bound) : "memory");
+            } else if (sharing == 2) {
+                bound_key = (int32_t)0x80000000;
+#pragma unroll
+                for (int e = 0; e < kSlots; e += 4) {
+                    int32_t b0, b1, b2, b3;
+                    asm volatile("ld.relaxed.gpu.global.v4.s32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(b0), "=r"(b1), "=r"(b2), "=r"(b3)
+                                 : "l"(my_bound + e)
+                                 : "memory");
+                    bound_key = max(max(bound_key, max(b0, b1)), max(b2, b3));
+                }
+            }
             // squared norms of this warp's columns, chunk after chunk; rows past the end of the cache get +inf
             // and never enter a list
             for (int li = lane;; li += 32) {
@@ -609,7 +631,14 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             tc_fence_before();
             mbar_arrive(&ctl->tmem_empty[acc]);
             flush(cnt);   // after the accumulator is released: the MMAs of the next tile can start meanwhile
-            if (top.s[KP - 1] < bound) atomicMin(my_bound, float_key(top.s[KP - 1]));
+            // publish this list where it changed
+            if (cnt > 0 && sharing == 1) {
+                if (top.s[KP - 1] < bound) atomicMin(my_bound, float_key(top.s[KP - 1]));
+            } else if (cnt > 0 && sharing == 2) {
+#pragma unroll
+                for (int e = 0; e < KP; ++e)
+                    if (top.s[e] <= bound) atomicMin(my_bound + ((list + e) & (KP - 1)), float_key(top.s[e]));
+            }
             __syncwarp();
         };
 
@@ -654,7 +683,8 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 top.reset();
                 for (int t = 0; t < sched.tiles && ok; ++t) {
                     const int col0 = sched.col_begin + t * sched.tile_w;
-                    select_tile(m_tile, col0, min(sched.tile_w, sched.col_end - col0));
+                    select_tile(m_tile, col0, min(sched.tile_w, sched.col_end - col0), MSUB == 1 ? sched.q * 2 + half : sched.q,
+                                sharing);
                 }
                 if (ok) emit_list(m_tile, MSUB == 1 ? sched.q * 2 + half : sched.q);
             }
@@ -662,7 +692,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             WorkItem it;
             sched.item(0, 0, 0, it);
             top.reset();
-            select_tile(it.m_tile, it.col0, it.w);
+            select_tile(it.m_tile, it.col0, it.w, it.list, 0);
             if (ok) emit_list(it.m_tile, it.list);
             if (ok && n_items > 1) {
                 sched.item(1, 0, 0, it);
@@ -857,7 +887,7 @@ fi_status_t launch_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, con
         attr_set = true;
     }
     // every bound starts at a huge finite value (0x7F7F7F7F as a float is 3.4e38)
-    if (cudaMemsetAsync(c->row_bound, 0x7F, ((size_t)batch_max + 256) * sizeof(int32_t), stream) != cudaSuccess) {
+    if (cudaMemsetAsync(c->row_bound, 0x7F, ((size_t)batch_max + 256) * KP * sizeof(int32_t), stream) != cudaSuccess) {
         set_error("cannot reset the row bounds");
         cudaGetLastError();
         return FI_ERR_CUDA;

@@ -173,7 +173,7 @@ struct fi_cache {
     uint8_t *slot_hit;
     float *tail_dump;        // partial sums of the tail tiles: [units][256 columns][256 rows], allocated on first need
     size_t tail_dump_units;
-    int32_t *row_bound;      // [max_batch + 256] per-query upper bound of the list_len-th best score, shared by all
+    int32_t *row_bound;      // [(max_batch + 256) x list_len] per-query slots whose maximum bounds the list_len-th best score, shared by all
                              // CTAs of a GEMM launch (order-preserving integer image of the float)
     fi::GemmPlan *plan_dev;  // written by the GEMM kernel, read by the finalize kernel
     int32_t *status_dev;     // device status word (bounded waits that ran out)
