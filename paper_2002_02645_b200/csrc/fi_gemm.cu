@@ -14,11 +14,13 @@
 //   256 queries: two 128-row MMAs share every cache-row stage, which halves the bytes the CTA pulls from L2
 //                per flop (the kernel is bound by L2-to-SM bandwidth, not by the tensor pipe); the two
 //                accumulators fill TMEM, so select and MMAs alternate; one epilogue warp per 32 rows.
-// Select: a thread owns one query row.  Scores of a 16-column chunk are formed with independent FMAs and
+// Select: a thread owns one query row.  Scores of two 16-column chunks are formed with independent FMAs and
 // tested against the row's current k-th best through one min-tree; the few that pass are parked in a small
 // per-thread queue in shared memory and inserted into the sorted register list once per tile, when all lanes
 // of the warp insert together (inserting on the spot makes the whole warp walk the insert code whenever any
-// one lane has a hit, which made the select 20x slower than the MMAs on short rows).
+// one lane has a hit, which made the select 20x slower than the MMAs on short rows).  What a tile's scan needs
+// from global memory (column norms, the row's shared bound) is fetched a tile ahead where the select is the
+// critical path.
 // Every wait is bounded: a wait that runs out sets the cache's status word and the CTA drains and returns.
 #include <cuda_bf16.h>
 
@@ -31,6 +33,7 @@ namespace {
 constexpr int kBlockK = 64;                       // bf16 elements per k-block: 128 bytes, one swizzle row
 constexpr int kMaxStages = 8;
 constexpr int kMaxTileN = 256;                    // cache rows per tile (MMA N), multiple of 16
+constexpr int kFirstTileN = 32;                   // cache rows of the short tile a long range opens with
 constexpr int kABytes = kTileM * kBlockK * 2;     // 16 KiB
 constexpr int kStageRegionBytes = 200 * 1024;     // operand ring; a stage is A (16 or 32 KiB) + B (tile width x 128 bytes)
 constexpr int kMaxEpiWarps = 8;
@@ -50,8 +53,9 @@ struct __align__(8) SmemCtl {
 constexpr int kEpiThreads = kMaxEpiWarps * 32;
 constexpr int kGemmThreads = 64 + kEpiThreads;
 constexpr int kNormSmemBytes = kMaxEpiWarps * kMaxTileN * 4;   // 256 floats per epilogue warp
-constexpr int kQueueCap = 8;                                    // pending candidates per epilogue thread
-constexpr int kQueueSmemBytes = kQueueCap * kEpiThreads * 8;    // scores + indices
+constexpr int kQueueCap = 7;                                    // pending candidates per epilogue thread
+constexpr int kQueueStride = kEpiThreads * 8;                   // bytes between a thread's slots: (score, column) pairs
+constexpr int kQueueSmemBytes = (kQueueCap + 1) * kQueueStride; // one more slot takes what does not fit
 constexpr int kGemmSmemBytes =
     1024 /*alignment slack*/ + kStageRegionBytes + kNormSmemBytes + kQueueSmemBytes + (int)sizeof(SmemCtl);
 
@@ -162,6 +166,8 @@ __device__ __forceinline__ int32_t float_key(float f) {
     return b >= 0 ? b : b ^ 0x7FFFFFFF;
 }
 __device__ __forceinline__ float key_float(int32_t k) { return __int_as_float(k >= 0 ? k : k ^ 0x7FFFFFFF); }
+// smallest of three (the compiler folds the pair into the three-input minimum of this architecture)
+__device__ __forceinline__ float fmin3(float a, float b, float c) { return fminf(fminf(a, b), c); }
 
 template <int KP>
 struct TopList {
@@ -206,9 +212,10 @@ struct Schedule {
     int cta, num_ctas, m_local, q, num_kb;
     long long n16;
     // ranges mode
-    int col_begin, col_end, tiles, tile_w, my_groups;
+    int col_begin, col_end, tiles, tile_w, first_w, my_groups;
 
-    __device__ __forceinline__ void setup(const GemmPlan &p, int cta_, int num_ctas_, long long n_entries, int num_kb_) {
+    __device__ __forceinline__ void setup(const GemmPlan &p, int cta_, int num_ctas_, long long n_entries, int num_kb_,
+                                          bool short_first_tile) {
         plan = p;
         cta = cta_;
         num_ctas = num_ctas_;
@@ -216,7 +223,7 @@ struct Schedule {
         n16 = (n_entries + 15) / 16;
         m_local = cta % p.mg;
         q = cta / p.mg;
-        col_begin = col_end = tiles = tile_w = my_groups = 0;
+        col_begin = col_end = tiles = tile_w = first_w = my_groups = 0;
         if (p.mode == 0 && p.m_tiles > 0 && p.range16 > 0 && q < p.parts) {
             long long b = (long long)q * p.range16, e = b + p.range16;
             if (e > n16) e = n16;
@@ -224,13 +231,30 @@ struct Schedule {
             col_begin = (int)(b * 16);
             col_end = (int)(e * 16);
             const int cols = col_end - col_begin;
-            tiles = (cols + kMaxTileN - 1) / kMaxTileN;
-            tile_w = tiles > 0 ? (((cols + tiles - 1) / tiles + 15) / 16) * 16 : 0;
+            // Where the select is the critical path (128-row tiles over short rows), long ranges open with a tile of
+            // only kFirstTileN rows.  A list that starts empty takes in nearly every column it sees, one insertion
+            // each; after a short first tile all lists of a query publish their first bounds, and the tiles that
+            // follow are scanned against a bound that already covers (number of lists x kFirstTileN / 2) cache rows
+            // instead of every list warming up on its own.  Elsewhere the extra tile would only lengthen the MMA
+            // pipeline's serial part.
+            first_w = short_first_tile && cols > 3 * kMaxTileN ? kFirstTileN : 0;
+            const int rest_tiles = (cols - first_w + kMaxTileN - 1) / kMaxTileN;
+            tile_w = rest_tiles > 0 ? (((cols - first_w + rest_tiles - 1) / rest_tiles + 15) / 16) * 16 : 0;
+            tiles = rest_tiles + (first_w ? 1 : 0);
             my_groups = m_local < p.m_tiles ? (p.m_tiles - m_local + p.mg - 1) / p.mg : 0;
         }
     }
     // widest tile this CTA will load (sizes the shared-memory stages)
     __device__ __forceinline__ int max_width() const { return plan.mode == 0 ? tile_w : kMaxTileN; }
+    // ranges mode: first cache row and width of this CTA's t-th tile
+    __device__ __forceinline__ int tile_col0(int t) const {
+        return col_begin + (first_w && t ? first_w + (t - 1) * tile_w : t * tile_w);
+    }
+    __device__ __forceinline__ int tile_width(int t) const {
+        if (first_w && t == 0) return first_w;
+        const int rest = col_end - tile_col0(t);
+        return rest < tile_w ? rest : tile_w;
+    }
     __device__ __forceinline__ int num_items() const {
         if (plan.m_tiles == 0 || n16 == 0) return 0;
         if (plan.mode == 0) return my_groups * tiles;
@@ -253,9 +277,8 @@ struct Schedule {
         it.dump_slot = 0;
         if (plan.mode == 0) {
             it.m_tile = g * plan.mg + m_local;
-            it.col0 = col_begin + t * tile_w;
-            const int rest = col_end - it.col0;
-            it.w = rest < tile_w ? rest : tile_w;
+            it.col0 = tile_col0(t);
+            it.w = tile_width(t);
             it.kb0 = 0;
             it.kb1 = num_kb;
             it.list = q;
@@ -308,8 +331,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char *stage_base = smem;
     float *norm_smem = reinterpret_cast<float *>(smem + kStageRegionBytes);
-    float *queue_s = reinterpret_cast<float *>(smem + kStageRegionBytes + kNormSmemBytes);
-    int32_t *queue_i = reinterpret_cast<int32_t *>(queue_s + kQueueCap * kEpiThreads);
+    unsigned char *queue_smem = smem + kStageRegionBytes + kNormSmemBytes;
     SmemCtl *ctl = reinterpret_cast<SmemCtl *>(smem + kStageRegionBytes + kNormSmemBytes + kQueueSmemBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -325,7 +347,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     }
     __syncthreads();
     Schedule sched;
-    sched.setup(ctl->plan, (int)blockIdx.x, (int)gridDim.x, n_entries, num_kb);
+    sched.setup(ctl->plan, (int)blockIdx.x, (int)gridDim.x, n_entries, num_kb, MSUB == 1 && num_kb <= 8);
     const GemmPlan &plan = sched.plan;
     const int n_items = sched.num_items();
     if (n_items == 0) return;   // whole CTA, before any barrier
@@ -388,10 +410,8 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             };
             if (plan.mode == 0) {
                 for (int g = 0; g < sched.my_groups && ok; ++g)
-                    for (int t = 0; t < sched.tiles && ok; ++t) {
-                        const int col0 = sched.col_begin + t * sched.tile_w;
-                        load_tile(g * plan.mg + sched.m_local, col0, min(sched.tile_w, sched.col_end - col0), 0, num_kb);
-                    }
+                    for (int t = 0; t < sched.tiles && ok; ++t)
+                        load_tile(g * plan.mg + sched.m_local, sched.tile_col0(t), sched.tile_width(t), 0, num_kb);
             } else {
                 for (int idx = 0; idx < n_items && ok; ++idx) {
                     WorkItem it;
@@ -457,7 +477,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             if (plan.mode == 0) {
                 for (int g = 0; g < sched.my_groups && ok; ++g)
                     for (int t = 0; t < sched.tiles && ok; ++t)
-                        mma_tile(min(sched.tile_w, sched.col_end - (sched.col_begin + t * sched.tile_w)), 0, num_kb);
+                        mma_tile(sched.tile_width(t), 0, num_kb);
             } else {
                 for (int idx = 0; idx < n_items && ok; ++idx) {
                     WorkItem it;
@@ -477,8 +497,8 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         const int row_in_tile = msub * kTileM + quarter * 32 + lane;
         const int te = threadIdx.x - 64;                  // 0..255, queue slot
         float *my_norm = norm_smem + ew * kMaxTileN;      // 256 floats: one buffer (256-row tiles) or two of 128
-        float *qs = queue_s + te;
-        int32_t *qi = queue_i + te;
+        // queue slots and norms are read and written through explicit shared-memory addresses
+        const uint32_t q_base = smem_u32(queue_smem) + (uint32_t)te * 8u;
         TopList<KP> top;
         bool ok = true;
 
@@ -495,142 +515,224 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         const int sharing = plan.mode != 0 || sched.tiles < 2 ? 0 : sched.tiles < 4 ? 1 : 2;
         float bound = __int_as_float(0x7F800000);
 
+        // slot r of this thread's queue
+        auto q_read = [&](int r, float &sc, int32_t &col) {
+            uint32_t a, b;
+            asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(a), "=r"(b) : "r"(q_base + (uint32_t)r * kQueueStride) : "memory");
+            sc = __uint_as_float(a);
+            col = (int32_t)b;
+        };
+        // append; what does not fit lands in the spare slot and is found again by rescanning the columns
+        auto q_push = [&](int &cnt, float sc, int32_t col) {
+            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(q_base + (uint32_t)min(cnt, kQueueCap) * kQueueStride),
+                         "r"(__float_as_uint(sc)), "r"(col)
+                         : "memory");
+            ++cnt;
+        };
         // insert the first n queued candidates of every lane, all lanes together
         auto flush = [&](int n) {
             const int rounds = __reduce_max_sync(0xFFFFFFFFu, n);
             for (int r = 0; r < rounds; ++r) {
                 if (r < n) {
-                    const float sc = qs[r * kEpiThreads];
-                    if (sc < top.s[KP - 1] && sc <= bound) top.insert(sc, qi[r * kEpiThreads]);
+                    float sc;
+                    int32_t col;
+                    q_read(r, sc, col);
+                    if (sc < top.s[KP - 1] && sc <= bound) top.insert(sc, col);
                 }
+            }
+        };
+        // the same for one lane on its own (other lanes idle meanwhile)
+        auto drain = [&](int n) {
+            for (int r = 0; r < n; ++r) {
+                float sc;
+                int32_t col;
+                q_read(r, sc, col);
+                if (sc < top.s[KP - 1] && sc <= bound) top.insert(sc, col);
             }
         };
 
         uint32_t tile_no = 0;
 
-        // scan one accumulator tile into the running list of this thread's row
-        auto select_tile = [&](int m_tile, int col0, int w, int list, int sharing) {
+        // What a tile's scan needs from global memory: the row's bound slots and the squared norms of the tile's
+        // columns.  With 128-row tiles the epilogue is the critical path, so both are fetched a tile ahead (the slots
+        // into registers before the previous tile's queue is drained, the norms by asynchronous copies into the
+        // other half of the norm buffer while the previous tile is scanned); only a CTA's first tile, and 256-row
+        // tiles (whose scan waits for the MMAs anyway and whose norms fill the buffer), fetch them on the spot.
+        // (long lists keep too many slots to hold them in registers across a drain: those are read on the spot)
+        constexpr bool kSlotsAhead = KP <= 8;
+        int32_t slot_regs[kSlots];   // raw slot values of the next tile's row (slot_regs[0] alone when one slot is shared)
+        bool fetched_ahead = false;
+
+        // the row's slots, read past L1 (other SMs lower them)
+        auto load_slots = [&](int m_tile, int sharing) {
+            const int32_t *my_bound = row_bound + (long long)(m_tile * kTileRows + row_in_tile) * kSlots;
+            if (sharing == 1) {
+                asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(slot_regs[0]) : "l"(my_bound) : "memory");
+            } else if (sharing == 2) {
+#pragma unroll
+                for (int e = 0; e < kSlots; e += 4)
+                    asm volatile("ld.relaxed.gpu.global.v4.s32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(slot_regs[e]), "=r"(slot_regs[e + 1]), "=r"(slot_regs[e + 2]), "=r"(slot_regs[e + 3])
+                                 : "l"(my_bound + e)
+                                 : "memory");
+            }
+        };
+        // the bound is the largest of the slots
+        auto slots_bound = [&](int sharing) -> int32_t {
+            if (sharing == 1) return slot_regs[0];
+            if (sharing != 2) return 0x7F7F7F7F;
+            int32_t key = (int32_t)0x80000000;
+#pragma unroll
+            for (int e = 0; e < kSlots; e += 4)
+                key = max(max(key, max(slot_regs[e], slot_regs[e + 1])), max(slot_regs[e + 2], slot_regs[e + 3]));
+            return key;
+        };
+        // squared norms of this warp's columns, chunk after chunk; rows past the end of the cache get +inf and
+        // never enter a list
+        // (a warp scans its chunks two at a time; an odd last chunk is paired with a chunk of +inf)
+        auto stage_norms = [&](float *nrm, int col0, int w, bool async) {
+            const int nch = (w - first + kStep - 1) / kStep;   // this warp's chunks
+            const float inf = __int_as_float(0x7F800000);
+            // four norms (16 bytes) per lane and round: a chunk is four lanes wide
+            for (int u = lane; u < ((nch + 1) >> 1) * 8; u += 32) {
+                const int c = first + (u >> 2) * kStep + (u & 3) * 4;
+                const uint32_t dst = smem_u32(nrm + u * 4);
+                const long long g = (long long)col0 + c;
+                if ((u >> 2) >= nch || g >= n_entries) {
+                    asm volatile("st.shared.v4.f32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "f"(inf) : "memory");
+                } else if (g + 3 < n_entries) {
+                    if (async) {
+                        asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(norms + g) : "memory");
+                    } else {
+                        const float4 v = __ldg(reinterpret_cast<const float4 *>(norms + g));
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+                                     : "memory");
+                    }
+                } else {
+                    // the cache ends inside these four columns
+                    for (int e = 0; e < 4; ++e) nrm[u * 4 + e] = g + e < n_entries ? __ldg(norms + g + e) : inf;
+                }
+            }
+        };
+
+        // scan one accumulator tile into the running list of this thread's row; (nx_m_tile, nx_col0, nx_w) is the
+        // tile this warp scans next (nx_w = 0: none)
+        auto select_tile = [&](int m_tile, int col0, int w, int list, int sharing, int nx_m_tile, int nx_col0, int nx_w,
+                               bool fresh_slots) {
             const uint32_t acc = tile_no % kAccBufs, acc_ph = (tile_no / kAccBufs) & 1;
             ++tile_no;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (acc + msub) * kMaxTileN;
             int32_t *my_bound = row_bound + (long long)(m_tile * kTileRows + row_in_tile) * kSlots;
             float *nrm = my_norm + acc * (kMaxTileN / 2);   // acc is 0 for 256-row tiles
-            // the row's slots, read past L1 (other SMs lower them); the bound is the largest of them
-            int32_t bound_key = 0x7F7F7F7F;
-            if (sharing == 1) {
-                asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(bound_key) : "l"(my_bound) : "memory");
-            } else if (sharing == 2) {
-                bound_key = (int32_t)0x80000000;
-#pragma unroll
-                for (int e = 0; e < kSlots; e += 4) {
-                    int32_t b0, b1, b2, b3;
-                    asm volatile("ld.relaxed.gpu.global.v4.s32 {%0, %1, %2, %3}, [%4];"
-                                 : "=r"(b0), "=r"(b1), "=r"(b2), "=r"(b3)
-                                 : "l"(my_bound + e)
-                                 : "memory");
-                    bound_key = max(max(bound_key, max(b0, b1)), max(b2, b3));
-                }
-            }
-            // squared norms of this warp's columns, chunk after chunk; rows past the end of the cache get +inf
-            // and never enter a list
-            for (int li = lane;; li += 32) {
-                const int c = first + (li >> 4) * kStep + (li & 15);
-                if (c - (li & 15) >= w) break;
-                nrm[li] = (long long)(col0 + c) < n_entries ? __ldg(norms + col0 + c) : __int_as_float(0x7F800000);
+            if (!fetched_ahead) {
+                load_slots(m_tile, sharing);
+                stage_norms(nrm, col0, w, false);
+            } else {
+                if (!kSlotsAhead) load_slots(m_tile, sharing);
+                asm volatile("cp.async.wait_all;" ::: "memory");
             }
             __syncwarp();
             // the whole warp takes the same decision, so its lanes stay together for the TMEM loads
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, status, 4));
             if (!ok) return;
             tc_fence_after();
+            if (fresh_slots) load_slots(m_tile, sharing);
+            const int32_t bound_key = slots_bound(sharing);
+            fetched_ahead = MSUB == 1 && nx_w > 0;
+            if (fetched_ahead) stage_norms(my_norm + (acc ^ 1) * (kMaxTileN / 2), nx_col0, nx_w, true);
             bound = key_float(bound_key);
             float thr = fminf(top.s[KP - 1], bound);   // pre-filter: nothing above it can enter the list
             int cnt = 0;
 
-            auto process = [&](const uint32_t (&v)[16], int c0, int li0) {
-                const float4 *n4 = reinterpret_cast<const float4 *>(nrm + li0);
-                const float4 na = n4[0], nb = n4[1], nc = n4[2], nd = n4[3];
-                const float nv[16] = {na.x, na.y, na.z, na.w, nb.x, nb.y, nb.z, nb.w,
-                                      nc.x, nc.y, nc.z, nc.w, nd.x, nd.y, nd.z, nd.w};
-                float sc[16];
+            const uint32_t nrm_addr = smem_u32(nrm);
+            const int nch = (w - first + kStep - 1) / kStep;   // this warp's chunks of 16 columns
+            const int npairs = (nch + 1) >> 1;
+
+            // Two chunks (32 columns) per step: all loads and the 32 score FMAs are independent, one min-tree
+            // decides whether any column can enter the list.  The rare rest is lane-local: only the groups of four
+            // columns that hold a passing score are walked, the passing columns are queued, and a lane whose queue
+            // overflows inserts what it had queued, tightens its threshold and walks the step again.
+            // TMEM loads of pair p; a missing second chunk reads the first again (its norms are +inf)
+            auto issue = [&](uint32_t (&v0)[16], uint32_t (&v1)[16], int p) {
+                const int ca = first + 2 * p * kStep;
+                const int cb = 2 * p + 1 < nch ? ca + kStep : ca;
+                __syncwarp();
+                tmem_ld16(taddr + ca, v0);
+                tmem_ld16(taddr + cb, v1);
+            };
+            // one register buffer: the loads of the next step are issued as soon as this step's scores are formed
+            // and are in flight while they are examined
+            uint32_t v0[16], v1[16];
+            if (npairs > 0) issue(v0, v1, 0);
+            for (int p = 0; p < npairs; ++p) {
+                const int ca = first + 2 * p * kStep;                 // first chunk of the pair
+                const int cb = ca + kStep;                            // second chunk (columns of +inf when past the tile)
+                float sc[32];
+                tmem_ld_wait(v0);
+                tmem_ld_wait(v1);
 #pragma unroll
-                for (int j = 0; j < 16; ++j) sc[j] = fmaf(-2.f, __uint_as_float(v[j]), nv[j]);
-                float m0 = fminf(fminf(sc[0], sc[1]), fminf(sc[2], sc[3]));
-                float m1 = fminf(fminf(sc[4], sc[5]), fminf(sc[6], sc[7]));
-                float m2 = fminf(fminf(sc[8], sc[9]), fminf(sc[10], sc[11]));
-                float m3 = fminf(fminf(sc[12], sc[13]), fminf(sc[14], sc[15]));
-                const float mn = fminf(fminf(m0, m1), fminf(m2, m3));
-                const int cnt0 = cnt;
-                if (mn <= thr) {
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        if (sc[j] <= thr) {
-                            if (cnt < kQueueCap) {
-                                qs[cnt * kEpiThreads] = sc[j];
-                                qi[cnt * kEpiThreads] = col0 + c0 + j;
-                            }
-                            ++cnt;
-                        }
-                    }
+                for (int q4 = 0; q4 < 8; ++q4) {
+                    float n0, n1, n2, n3;
+                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                 : "=f"(n0), "=f"(n1), "=f"(n2), "=f"(n3)
+                                 : "r"(nrm_addr + (uint32_t)(p * 32 + q4 * 4) * 4u));
+                    const uint32_t *v = q4 < 4 ? &v0[q4 * 4] : &v1[(q4 - 4) * 4];
+                    sc[q4 * 4 + 0] = fmaf(-2.f, __uint_as_float(v[0]), n0);
+                    sc[q4 * 4 + 1] = fmaf(-2.f, __uint_as_float(v[1]), n1);
+                    sc[q4 * 4 + 2] = fmaf(-2.f, __uint_as_float(v[2]), n2);
+                    sc[q4 * 4 + 3] = fmaf(-2.f, __uint_as_float(v[3]), n3);
                 }
-                if (__any_sync(0xFFFFFFFFu, cnt > kQueueCap)) {
-                    // a queue overflowed inside this chunk: insert what was queued before it (all lanes together),
-                    // then queue this chunk again against the tighter threshold; only if that overflows too (lists
-                    // still filling up) is it inserted column by column.  Arrival order, hence the tie order, is kept.
-                    flush(cnt0);
-                    thr = fminf(top.s[KP - 1], bound);
-                    cnt = 0;
-                    if (mn <= thr) {
+                if (p + 1 < npairs) issue(v0, v1, p + 1);
+                float gm[8];
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            if (sc[j] <= thr) {
-                                if (cnt < kQueueCap) {
-                                    qs[cnt * kEpiThreads] = sc[j];
-                                    qi[cnt * kEpiThreads] = col0 + c0 + j;
+                for (int g = 0; g < 8; ++g) gm[g] = fminf(fmin3(sc[4 * g], sc[4 * g + 1], sc[4 * g + 2]), sc[4 * g + 3]);
+                const float mn = fminf(fmin3(gm[0], gm[1], gm[2]), fminf(fmin3(gm[3], gm[4], gm[5]), fminf(gm[6], gm[7])));
+                if (mn <= thr) {
+                    const int cnt0 = cnt;
+                    auto walk = [&]() {
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            if (gm[g] <= thr) {
+#pragma unroll
+                                for (int jj = 0; jj < 4; ++jj) {
+                                    const int j = 4 * g + jj;
+                                    if (sc[j] <= thr) q_push(cnt, sc[j], col0 + (j < 16 ? ca + j : cb + j - 16));
                                 }
-                                ++cnt;
                             }
                         }
+                    };
+                    // no threshold yet (the list is not full and no bound is known): every column passes, so
+                    // queueing them would only overflow
+                    bool direct = !(thr < __int_as_float(0x7F800000));
+                    int pending = cnt0;
+                    if (!direct) {
+                        walk();
+                        if (cnt > kQueueCap) {
+                            drain(cnt0);
+                            pending = 0;
+                            thr = fminf(top.s[KP - 1], bound);
+                            cnt = 0;
+                            walk();
+                            direct = cnt > kQueueCap;   // still too many: the list is filling up
+                        }
                     }
-                    if (__any_sync(0xFFFFFFFFu, cnt > kQueueCap)) {
+                    if (direct) {
+                        // insert column by column; arrival order, hence the tie order, is kept
+                        drain(pending);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (sc[j] < top.s[KP - 1] && sc[j] <= bound) top.insert(sc[j], col0 + c0 + j);
+                        for (int j = 0; j < 32; ++j)
+                            if (sc[j] < top.s[KP - 1] && sc[j] <= bound) top.insert(sc[j], col0 + (j < 16 ? ca + j : cb + j - 16));
                         cnt = 0;
                         thr = fminf(top.s[KP - 1], bound);
                     }
                 }
-            };
-
-            // two register buffers: the TMEM load of the next chunk is in flight while this one is scanned
-            uint32_t va[16], vb[16];
-            int c0 = first, li0 = 0;
-            if (c0 < w) {
-                __syncwarp();
-                tmem_ld16(taddr + c0, va);
             }
-            while (c0 < w) {
-                tmem_ld_wait(va);
-                if (c0 + kStep < w) {
-                    __syncwarp();
-                    tmem_ld16(taddr + c0 + kStep, vb);
-                }
-                process(va, c0, li0);
-                c0 += kStep;
-                li0 += 16;
-                if (c0 >= w) break;
-                tmem_ld_wait(vb);
-                if (c0 + kStep < w) {
-                    __syncwarp();
-                    tmem_ld16(taddr + c0 + kStep, va);
-                }
-                process(vb, c0, li0);
-                c0 += kStep;
-                li0 += 16;
-            }
+            __syncwarp();
             tc_fence_before();
             mbar_arrive(&ctl->tmem_empty[acc]);
-            flush(cnt);   // after the accumulator is released: the MMAs of the next tile can start meanwhile
+            if (kSlotsAhead && fetched_ahead) load_slots(nx_m_tile, sharing);   // in flight while the queue is drained
+            // after the accumulator is released: the MMAs of the next tile can start meanwhile
+            if (__any_sync(0xFFFFFFFFu, cnt > 0)) flush(cnt);
             // publish this list where it changed
             if (cnt > 0 && sharing == 1) {
                 if (top.s[KP - 1] < bound) atomicMin(my_bound, float_key(top.s[KP - 1]));
@@ -682,9 +784,12 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 const int m_tile = g * plan.mg + sched.m_local;
                 top.reset();
                 for (int t = 0; t < sched.tiles && ok; ++t) {
-                    const int col0 = sched.col_begin + t * sched.tile_w;
-                    select_tile(m_tile, col0, min(sched.tile_w, sched.col_end - col0), MSUB == 1 ? sched.q * 2 + half : sched.q,
-                                sharing);
+                    const bool last_t = t + 1 == sched.tiles;
+                    const int nx_t = last_t ? 0 : t + 1;
+                    const int nx_w = last_t && g + 1 == sched.my_groups ? 0 : sched.tile_width(nx_t);
+                    // while the lists of a query are young their bounds move fast: read the slots as late as possible
+                    select_tile(m_tile, sched.tile_col0(t), sched.tile_width(t), MSUB == 1 ? sched.q * 2 + half : sched.q,
+                                sharing, last_t ? m_tile + plan.mg : m_tile, sched.tile_col0(nx_t), nx_w, t < 3);
                 }
                 if (ok) emit_list(m_tile, MSUB == 1 ? sched.q * 2 + half : sched.q);
             }
@@ -692,7 +797,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             WorkItem it;
             sched.item(0, 0, 0, it);
             top.reset();
-            select_tile(it.m_tile, it.col0, it.w, it.list, 0);
+            select_tile(it.m_tile, it.col0, it.w, it.list, 0, 0, 0, 0, false);
             if (ok) emit_list(it.m_tile, it.list);
             if (ok && n_items > 1) {
                 sched.item(1, 0, 0, it);
