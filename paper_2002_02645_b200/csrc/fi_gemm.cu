@@ -6,8 +6,9 @@
 // accumulator tiles back from TMEM (one query row per thread) and keeps the `list_len` smallest scores of its
 // row in registers.  The exact distances of those few candidates are recomputed afterwards (finalize_kernel).
 //
-// Roles inside a CTA of 320 threads: warp 0 = TMA producer (one lane), warp 1 = TMEM owner and MMA issuer (one
-// lane), warps 2..9 = epilogue.  Shared-memory stages are handed over with mbarriers.  Two tile heights:
+// Roles inside a CTA of 384 threads (three warpgroups): warp 0 = TMA producer (one lane), warp 1 = TMEM owner and
+// MMA issuer (one lane), warps 2..3 idle, warps 4..11 = epilogue.  Warpgroup 0 hands most of its registers to the
+// epilogue warpgroups (setmaxnreg).  Shared-memory stages are handed over with mbarriers.  Two tile heights:
 //   128 queries: accumulator double-buffered in TMEM (2 x 256 columns), so the select of one tile overlaps
 //                the MMAs of the next; two epilogue warps per 32 rows, each taking every other 16-column chunk
 //                and keeping its own list.  For short rows (few k-blocks per tile), where the select dominates.
@@ -51,7 +52,15 @@ struct __align__(8) SmemCtl {
 };
 
 constexpr int kEpiThreads = kMaxEpiWarps * 32;
-constexpr int kGemmThreads = 64 + kEpiThreads;
+constexpr int kRoleThreads = 128;                  // warpgroup 0: TMA producer, MMA issuer, two idle warps
+constexpr int kGemmThreads = kRoleThreads + kEpiThreads;
+// Register split between the warpgroups (setmaxnreg): the kernel is launched with kLaunchRegs per thread, warpgroup
+// 0 gives back all but kRoleRegs, the two epilogue warpgroups grow to kEpiRegs.  The shares must fit the launch's
+// total, or the growing warps would wait for ever: checked here and again by the host against the compiled kernel.
+constexpr int kLaunchRegs = 168;
+constexpr int kRoleRegs = 56;
+constexpr int kEpiRegs = 224;
+static_assert(kRoleThreads * kRoleRegs + kEpiThreads * kEpiRegs <= kGemmThreads * kLaunchRegs, "register shares exceed the launch's total");
 constexpr int kNormSmemBytes = kMaxEpiWarps * kMaxTileN * 4;   // 256 floats per epilogue warp
 constexpr int kQueueCap = 7;                                    // pending candidates per epilogue thread
 constexpr int kQueueStride = kEpiThreads * 8;                   // bytes between a thread's slots: (score, column) pairs
@@ -378,6 +387,9 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
+    // Warpgroup 0 (all four warps at this one instruction) gives registers back before its warps take their roles;
+    // the epilogue warpgroups claim theirs.
+    if (warp < kRoleThreads / 32) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRoleRegs));
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -486,16 +498,17 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 }
             }
         }
-    } else {
+    } else if (warp >= kRoleThreads / 32) {
         // ------------------------------------------------------------ epilogue: per-row select
-        const int ew = warp - 2;                          // 0..7
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kEpiRegs));
+        const int ew = warp - kRoleThreads / 32;          // 0..7
         const int quarter = warp & 3;                     // TMEM lanes this warp may read: 32*quarter .. +31
         const int msub = MSUB == 2 ? (ew >> 2) : 0;       // which 128-row MMA this warp drains
         const int half = MSUB == 1 ? (ew >> 2) : 0;       // 128-row tiles: which 16-column chunks (even / odd)
         constexpr int kStep = MSUB == 1 ? 32 : 16;        // distance between this warp's chunks
         const int first = half * 16;
         const int row_in_tile = msub * kTileM + quarter * 32 + lane;
-        const int te = threadIdx.x - 64;                  // 0..255, queue slot
+        const int te = threadIdx.x - kRoleThreads;        // 0..255, queue slot
         float *my_norm = norm_smem + ew * kMaxTileN;      // 256 floats: one buffer (256-row tiles) or two of 128
         // queue slots and norms are read and written through explicit shared-memory addresses
         const uint32_t q_base = smem_u32(queue_smem) + (uint32_t)te * 8u;
@@ -978,17 +991,38 @@ fi_status_t encode_bf16_map(CUtensorMap *map, const void *base, uint64_t rows, u
     return FI_OK;
 }
 
+// One-time set-up of a kernel instantiation: shared-memory reservation, and the proof that the register shares its
+// warpgroups claim (setmaxnreg) fit what a launch of kGemmThreads threads is given.  Registers are handed out in
+// units of 8 per thread; a kernel compiled to fewer registers than the split assumes must never be launched.
+template <typename Kern>
+fi_status_t prepare_gemm_kernel(Kern kern, const char *what) {
+    cudaFuncAttributes attr;
+    if (cudaFuncGetAttributes(&attr, kern) != cudaSuccess) {
+        set_error("cannot query the attributes of the %s", what);
+        cudaGetLastError();
+        return FI_ERR_CUDA;
+    }
+    const int allocated = (attr.numRegs + 7) / 8 * 8;
+    if (allocated * kGemmThreads < kRoleThreads * kRoleRegs + kEpiThreads * kEpiRegs) {
+        set_error("%s: compiled to %d registers per thread, too few for its register split", what, attr.numRegs);
+        return FI_ERR_UNSUPPORTED;
+    }
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) != cudaSuccess) {
+        set_error("cannot reserve %d bytes of shared memory for the %s", kGemmSmemBytes, what);
+        cudaGetLastError();
+        return FI_ERR_CUDA;
+    }
+    return FI_OK;
+}
+
 template <int KP, int MSUB>
 fi_status_t launch_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, const int32_t *count_dev, bool tail_possible,
                       cudaStream_t stream) {
     static bool attr_set = false;
     auto kern = gemm_select_kernel<KP, MSUB>;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) != cudaSuccess) {
-            set_error("cannot reserve %d bytes of shared memory for the distance GEMM", kGemmSmemBytes);
-            cudaGetLastError();
-            return FI_ERR_CUDA;
-        }
+        const fi_status_t ps = prepare_gemm_kernel(kern, "distance GEMM");
+        if (ps != FI_OK) return ps;
         attr_set = true;
     }
     // every bound starts at a huge finite value (0x7F7F7F7F as a float is 3.4e38)
@@ -1136,11 +1170,8 @@ fi_status_t launch_gemm_project(fi_cache *w, const void *queries_compact, int64_
     static bool attr_set = false;
     auto kern = gemm_select_kernel<8, 2>;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) != cudaSuccess) {
-            set_error("cannot reserve %d bytes of shared memory for the projection", kGemmSmemBytes);
-            cudaGetLastError();
-            return FI_ERR_CUDA;
-        }
+        const fi_status_t ps = prepare_gemm_kernel(kern, "projection GEMM");
+        if (ps != FI_OK) return ps;
         attr_set = true;
     }
     kern<<<w->sm_count, kGemmThreads, kGemmSmemBytes, stream>>>(tq, w->tmap_rows64, w->tmap_rows16, w->norms,
