@@ -100,6 +100,9 @@ def test_stream_path_large_dim_reads_queries_in_place():
     (3000, 4096, 64, 13),      # list length 16, deep K
     (2500, 136, 2200, 29),     # 18 query tiles (two groups), list length 32
     (9990, 4096, 900, 5),      # 4 x 40 tiles of 256 x 256 on 148 SMs: one full tile per CTA plus a tail cut along K
+    (12345, 256, 2000, 5),     # short rows, 16 query tiles x 9 long ranges: short first tile, bounds fetched a tile ahead
+    (20011, 512, 1100, 10),    # the same with list length 16 (bound slots read on the spot), ragged N and M
+    (9000, 320, 2048, 1),      # the same with list length 4, K = 5 blocks
 ])
 def test_gemm_path(n, d, b, k):
     w = dg.single_layer(name="t", n_cache=n, n_query=b, dim=d, num_classes=9, dtype="bf16", sigma=0.6, k=k, seed=5)
