@@ -17,6 +17,13 @@ namespace {
 constexpr int kFinThreads = 256;
 constexpr int kFinWarps = kFinThreads / 32;
 
+// order-preserving integer image of a float (compares like the float, so an integer minimum is a float minimum)
+__device__ __forceinline__ int32_t score_key(float f) {
+    const int32_t b = __float_as_int(f);
+    return b >= 0 ? b : b ^ 0x7FFFFFFF;
+}
+__device__ __forceinline__ float key_score(int32_t k) { return __int_as_float(k >= 0 ? k : k ^ 0x7FFFFFFF); }
+
 struct FinalizeParams {
     const void *X;
     const int32_t *labels;
@@ -85,7 +92,7 @@ __global__ void __launch_bounds__(kFinThreads) finalize_kernel(FinalizeParams p)
     __shared__ float cand_s[kMaxK];
     __shared__ float cand_d[kMaxK];
     __shared__ int32_t cand_i[kMaxK];
-    __shared__ float red_s[kFinWarps];
+    __shared__ int32_t red_k[kFinWarps];
     __shared__ int32_t red_i[kFinWarps];
 
     const int count = p.count_dev ? min(*p.count_dev, p.batch_max) : p.batch_max;
@@ -101,53 +108,45 @@ __global__ void __launch_bounds__(kFinThreads) finalize_kernel(FinalizeParams p)
     if (want > kMaxK) want = kMaxK;
     const float kInf = __int_as_float(0x7F800000);
 
-    // ---- merge: repeatedly take the smallest (score, index) pair above the previous pick
-    float prev_s = -kInf;
+    // ---- merge: repeatedly take the smallest (score, index) pair above the previous pick.  Scores are compared
+    // through their order-preserving integer images, so a warp's minimum is two warp-wide integer reductions
+    // (score image, then index among the lanes that hold that score) instead of a shuffle tree.
+    int32_t prev_k = (int32_t)0x80000000;
     int prev_i = -1;
     int cand_n = 0;
     for (int r = 0; r < want; ++r) {
-        float best_s = kInf;
+        int32_t best_k = 0x7FFFFFFF;
         int best_i = 0x7FFFFFFF;
         for (int e = tid; e < entries; e += kFinThreads) {
-            float s = ps[e];
-            int i = pi[e];
+            const int i = pi[e];
             if (i < 0 || i >= p.n_entries) continue;   // empty slot (an index past the cache cannot occur; never follow one)
-            bool above = r == 0 || pair_less(prev_s, prev_i, s, i);
-            if (above && pair_less(s, i, best_s, best_i)) {
-                best_s = s;
+            const int32_t k = score_key(ps[e]);
+            const bool above = r == 0 || k > prev_k || (k == prev_k && i > prev_i);
+            if (above && (k < best_k || (k == best_k && i < best_i))) {
+                best_k = k;
                 best_i = i;
             }
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            float os = __shfl_xor_sync(0xFFFFFFFFu, best_s, o);
-            int oi = __shfl_xor_sync(0xFFFFFFFFu, best_i, o);
-            if (pair_less(os, oi, best_s, best_i)) {
-                best_s = os;
-                best_i = oi;
-            }
-        }
+        int32_t mk = __reduce_min_sync(0xFFFFFFFFu, best_k);
+        int mi = __reduce_min_sync(0xFFFFFFFFu, best_k == mk ? best_i : 0x7FFFFFFF);
         if (lane == 0) {
-            red_s[warp] = best_s;
-            red_i[warp] = best_i;
+            red_k[warp] = mk;
+            red_i[warp] = mi;
         }
         __syncthreads();
-        best_s = red_s[0];
-        best_i = red_i[0];
-#pragma unroll
-        for (int w = 1; w < kFinWarps; ++w)
-            if (pair_less(red_s[w], red_i[w], best_s, best_i)) {
-                best_s = red_s[w];
-                best_i = red_i[w];
-            }
+        // every warp combines the warps' minima the same way
+        best_k = lane < kFinWarps ? red_k[lane] : 0x7FFFFFFF;
+        best_i = lane < kFinWarps ? red_i[lane] : 0x7FFFFFFF;
+        mk = __reduce_min_sync(0xFFFFFFFFu, best_k);
+        mi = __reduce_min_sync(0xFFFFFFFFu, best_k == mk ? best_i : 0x7FFFFFFF);
         __syncthreads();
-        if (best_i == 0x7FFFFFFF) break;   // lists exhausted
+        if (mi == 0x7FFFFFFF) break;   // lists exhausted
         if (tid == 0) {
-            cand_s[r] = best_s;
-            cand_i[r] = best_i;
+            cand_s[r] = key_score(mk);
+            cand_i[r] = mi;
         }
-        prev_s = best_s;
-        prev_i = best_i;
+        prev_k = mk;
+        prev_i = mi;
         cand_n = r + 1;
     }
     __syncthreads();
