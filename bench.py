@@ -529,7 +529,7 @@ def run_kmeans(args):
                         sigma=0.5, k=1, seed=0)
     st = w.stages[0]
     pts, labs = to_dev(st.cache_vecs, dev), torch.from_numpy(st.cache_labels).to(dev)
-    cache = fb.FreezeCache(dim=d, capacity=clusters, num_classes=10, k=1, dtype=fb.FI_BF16, max_batch=8192)
+    cache = fb.FreezeCache(dim=d, capacity=clusters, num_classes=10, k=1, dtype=fb.FI_BF16, max_batch=n)
     cache.insert(to_dev(st.queries, dev), torch.zeros(clusters, dtype=torch.int32, device=dev))
     for _ in range(max(args.warmup, 3)):
         cache.kmeans_step(pts, labs)

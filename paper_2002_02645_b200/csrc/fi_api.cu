@@ -62,6 +62,7 @@ void free_all(fi_cache *c) {
     cudaFree(c->tail_dump);
     cudaFree(c->calib_acc);
     cudaFree(c->km_dist);
+    cudaFree(c->km_partial);
     cudaFree(c->status_dev);
     cudaFree(c->h2d_stage);
     if (c->copy_ev) {

@@ -179,6 +179,8 @@ struct fi_cache {
     int32_t *status_dev;     // device status word (bounded waits that ran out)
     int32_t *calib_acc;      // [2] threshold calibration: max wrong confidence (bit pattern), wrong count
     float *km_dist;          // [max_batch] k-means assignment scratch: nearest distances of one batch (unused output)
+    float *km_partial;       // [size x segments x dim] k-means update: per-segment sums of the points of each cluster
+    size_t km_partial_elems; // floats allocated there (grown on demand)
     // staging for the host-buffer entry points (allocated on first use)
     void *h2d_stage;
     size_t h2d_stage_bytes;
@@ -236,7 +238,7 @@ fi_status_t launch_wrong_max(const int32_t *label, const float *conf, const int3
                              cudaStream_t stream);
 
 // k-means update step (means, counts, majority label and its share) for the centres held in `c`
-fi_status_t launch_kmeans_update(const fi_cache *c, const void *points, int64_t ld, const int32_t *point_labels,
+fi_status_t launch_kmeans_update(fi_cache *c, const void *points, int64_t ld, const int32_t *point_labels,
                                  const int32_t *assign, int64_t n, void *new_centres, int32_t *counts,
                                  int32_t *majority, float *fraction, cudaStream_t stream);
 
