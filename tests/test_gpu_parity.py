@@ -139,6 +139,26 @@ def test_kmeans_entries_weights_and_l2_metric():
     check_case(w.stages[0], k=4, num_classes=10, rule=fo.RULE_DIST_LE, path=fb.FI_PATH_GEMM, metric=1, weights=frac)
 
 
+@pytest.mark.parametrize("n,d,b,k,rule,metric,weighted", [
+    (3000, 64, 8200, 5, fo.RULE_CONF_GT, 0, False),     # the paper's vote, several labels among the neighbours
+    (200, 1024, 9000, 1, fo.RULE_CONF_GT, 1, True),     # k-means cache: k = 1, weights, L2 metric
+    (1500, 200, 8500, 13, fo.RULE_DIST_LE, 0, True),    # list length 16, distance rule
+    (700, 136, 8192, 29, fo.RULE_CONF_GT, 0, False),    # too many candidate entries for a warp: CTA per query
+    (200, 1024, 8200, 29, fo.RULE_CONF_GT, 0, False),   # 32 candidates per query: every lane of the warp holds one
+])
+def test_large_batches_of_short_rows(n, d, b, k, rule, metric, weighted):
+    """Batches of 8,192 and more against rows of at most 8 KiB are finished one query per warp."""
+    w = dg.single_layer(name="t", n_cache=n, n_query=b, dim=d, num_classes=7, dtype="bf16", sigma=0.6, k=k, seed=21)
+    weights = np.random.default_rng(3).uniform(0.3, 1.0, n).astype(np.float32) if weighted else None
+    check_case(w.stages[0], k=k, num_classes=7, rule=rule, path=fb.FI_PATH_GEMM, metric=metric, weights=weights)
+
+
+def test_large_batch_fp32_streaming_lists():
+    """The same finish on the streaming kernel's candidate lists (fp32 cache, exact distances, no re-ranking)."""
+    w = dg.single_layer(name="t", n_cache=300, n_query=8300, dim=32, num_classes=5, dtype="f32", sigma=0.5, k=3, seed=22)
+    check_case(w.stages[0], k=3, num_classes=5, rule=fo.RULE_CONF_GT, path=fb.FI_PATH_STREAM)
+
+
 # ------------------------------------------------------------------ degenerate cases
 
 def test_empty_cache_k_above_size_and_zero_batch():
