@@ -6,6 +6,8 @@
 // apply the confidence heuristic of Sec. 3 (S_i = m_i/k, C_i = S_i * sum_j w_j/d_j, arg-max) and the hit rule of
 // Pseudocode 1.
 //
+// finalize_rows_kernel: the same finish, one query per warp, for large batches of short rows.
+//
 // compact_kernel (one CTA): warp-ballot stream compaction of the misses, order kept (Sec. 5, rebuilding the
 // batch after each layer), and the scatter of (label, confidence, stage) for the requests frozen here.
 #include "fi_internal.cuh"
