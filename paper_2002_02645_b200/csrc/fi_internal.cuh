@@ -85,6 +85,17 @@ __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entrie
             return p;
         }
     }
+    // Few cache rows (one tile spans them all) under many query tiles, e.g. assigning points to k-means centres:
+    // cutting the rows into ranges would leave tiles a few rows wide, which the MMAs run at a fraction of their
+    // rate while every CTA re-reads the query tiles.  The query tiles are dealt round-robin to all CTAs instead.
+    if (n16 <= 16 && p.m_tiles >= num_ctas / 2) {
+        p.mg = p.m_tiles < num_ctas ? p.m_tiles : num_ctas;
+        p.groups = (p.m_tiles + p.mg - 1) / p.mg;
+        p.parts = 1;
+        p.range16 = (int32_t)n16;
+        p.lists = tile_m == kTileM ? 2 : 1;
+        return p;
+    }
     // Group size: the fewest MMA columns per CTA in total, except that on long ranges a larger group within 3 % of
     // that minimum is preferred: it means fewer, longer ranges, hence fewer candidate lists per query to warm up
     // and to merge, and more CTAs streaming the same cache rows at the same time.

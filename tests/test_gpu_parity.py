@@ -145,6 +145,8 @@ def test_kmeans_entries_weights_and_l2_metric():
     (1500, 200, 8500, 13, fo.RULE_DIST_LE, 0, True),    # list length 16, distance rule
     (700, 136, 8192, 29, fo.RULE_CONF_GT, 0, False),    # too many candidate entries for a warp: CTA per query
     (200, 1024, 8200, 29, fo.RULE_CONF_GT, 0, False),   # 32 candidates per query: every lane of the warp holds one
+    (200, 1024, 19000, 1, fo.RULE_CONF_GT, 1, True),    # 75 query tiles on one cache-row tile: dealt round-robin to the CTAs
+    (250, 64, 9500, 5, fo.RULE_CONF_GT, 0, False),      # the same with 128-query tiles (two lists per query)
 ])
 def test_large_batches_of_short_rows(n, d, b, k, rule, metric, weighted):
     """Batches of 8,192 and more against rows of at most 8 KiB are finished one query per warp."""
