@@ -112,7 +112,50 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
     int32_t prev_k = (int32_t)0x80000000;
     int prev_i = -1;
     int cand_n = 0;
-    for (int r = 0; r < want; ++r) {
+    // The distance GEMM leaves every list sorted by (score, index).  Up to 64 such lists are merged by warp 0 alone,
+    // lane l holding the heads of lists l and l + 32: a round is two warp-wide integer minima and one lane stepping
+    // its list, without any CTA-wide barrier.
+    __shared__ int32_t cand_n_sh;
+    const bool head_merge = p.refine != 0 && parts <= 64;
+    if (head_merge) {
+        if (warp == 0) {
+            auto head = [&](int list, int h, int32_t &k, int32_t &i) {
+                k = 0x7FFFFFFF;
+                i = 0x7FFFFFFF;
+                if (list < parts && h < list_len) {
+                    const int ii = pi[list * list_len + h];
+                    if (ii >= 0 && ii < p.n_entries) {   // else the list has ended (an index past the cache cannot occur; never follow one)
+                        k = score_key(ps[list * list_len + h]);
+                        i = ii;
+                    }
+                }
+            };
+            int h0 = 0, h1 = 0;
+            int32_t k0, i0, k1, i1;
+            head(lane, 0, k0, i0);
+            head(lane + 32, 0, k1, i1);
+            for (int r = 0; r < want; ++r) {
+                const bool lower = k0 < k1 || (k0 == k1 && i0 < i1);
+                const int32_t bk = lower ? k0 : k1, bi = lower ? i0 : i1;
+                const int32_t mk = __reduce_min_sync(0xFFFFFFFFu, bk);
+                const int32_t mi = __reduce_min_sync(0xFFFFFFFFu, bk == mk ? bi : 0x7FFFFFFF);
+                if (mi == 0x7FFFFFFF) break;   // lists exhausted
+                if (bk == mk && bi == mi) {    // a cache row sits in one list only: exactly one lane
+                    if (lower) head(lane, ++h0, k0, i0);
+                    else head(lane + 32, ++h1, k1, i1);
+                }
+                if (lane == 0) {
+                    cand_s[r] = key_score(mk);
+                    cand_i[r] = mi;
+                }
+                cand_n = r + 1;
+            }
+            if (lane == 0) cand_n_sh = cand_n;
+        }
+        __syncthreads();
+        cand_n = cand_n_sh;
+    }
+    for (int r = 0; r < want && !head_merge; ++r) {
         int32_t best_k = 0x7FFFFFFF;
         int best_i = 0x7FFFFFFF;
         for (int e = tid; e < entries; e += kFinThreads) {
