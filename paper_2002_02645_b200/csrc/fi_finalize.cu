@@ -95,6 +95,8 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
     __shared__ float cand_s[kMaxK];
     __shared__ float cand_d[kMaxK];
     __shared__ int32_t cand_i[kMaxK];
+    __shared__ int32_t cand_lab[kMaxK];
+    __shared__ float cand_w[kMaxK];
     __shared__ int32_t red_k[kFinWarps];
     __shared__ int32_t red_i[kFinWarps];
 
@@ -192,6 +194,11 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
     }
     __syncthreads();
 
+    // labels and weights of the candidates, fetched side by side while the distances are recomputed
+    if (tid < cand_n) {
+        cand_lab[tid] = p.labels[cand_i[tid]];
+        cand_w[tid] = p.weights[cand_i[tid]];
+    }
     // ---- exact distances of the candidates
     if (p.refine) {
         const int64_t qr = p.row_idx ? (int64_t)p.row_idx[b] : (int64_t)b;
@@ -224,24 +231,24 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
     // ---- order by (distance, index), vote, hit
     if (tid == 0) {
         for (int a = 1; a < cand_n; ++a) {
-            float d = cand_d[a];
-            int i = cand_i[a];
+            const float d = cand_d[a], w = cand_w[a];
+            const int i = cand_i[a], l = cand_lab[a];
             int pos = a;
             while (pos > 0 && pair_less(d, i, cand_d[pos - 1], cand_i[pos - 1])) {
                 cand_d[pos] = cand_d[pos - 1];
                 cand_i[pos] = cand_i[pos - 1];
+                cand_lab[pos] = cand_lab[pos - 1];
+                cand_w[pos] = cand_w[pos - 1];
                 --pos;
             }
             cand_d[pos] = d;
             cand_i[pos] = i;
+            cand_lab[pos] = l;
+            cand_w[pos] = w;
         }
         const int k_eff = cand_n < p.k ? cand_n : p.k;
-        int32_t lab[kMaxK];
-        float wgt[kMaxK];
-        for (int j = 0; j < k_eff; ++j) {
-            lab[j] = p.labels[cand_i[j]];
-            wgt[j] = p.weights[cand_i[j]];
-        }
+        const int32_t *lab = cand_lab;
+        const float *wgt = cand_w;
         int32_t best_label = -1;
         float best_c = 0.f, best_dwin = 0.f;
         int best_m = 0;
