@@ -11,7 +11,14 @@ entry point of the C ABI (pinned host activations copied in, results copied out,
 every rank holds its own caches and its own batch (the look-ups of different requests are independent, so
 ranks never exchange data): weak scaling.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg5] [--impl ours|reference]
+The default run (config 2, one GPU) also measures, in the same process, the configurations the two numeric targets
+sit on and puts them into the same JSON line under "targets": config 3 (tensor-core bound), config 5 at batch 1, 4
+and 16 (HBM bound, device-timed latency percentiles) and config 4's per-stage rates, each with its own clock record.
+
+`--gpus N` with N > 1 and no WORLD_SIZE in the environment starts the N ranks itself (torch.distributed.run, one
+process per GPU, rendezvous on 127.0.0.1); started under torchrun it uses the ranks it is given.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg4|cfg5|...] [--impl ours|reference]
 """
 from __future__ import annotations
 
@@ -50,8 +57,9 @@ def load_peaks():
 
 
 def captured_traffic(kernel: str, workload: str):
-    """DRAM bytes per launch of `kernel` on `workload` from the committed ncu summary, or None when there is no
-    capture or the kernel's source has changed since (the line carries the source file's sha256)."""
+    """(DRAM bytes per launch of `kernel` on `workload` from the committed ncu summary, where the figure comes from);
+    the figure is None when there is no capture or the kernel's source has changed since (the summary line carries the
+    source file's sha256).  Nothing is measured here: a run under a profiler is never a bench run."""
     import hashlib
     src = {"gemm_select_kernel": "fi_gemm.cu", "stream_lookup_kernel": "fi_stream.cu"}.get(kernel)
     try:
@@ -62,10 +70,11 @@ def captured_traffic(kernel: str, workload: str):
                 parts = line.split()
                 if len(parts) >= 4 and not line.startswith("#") and parts[0] == kernel and parts[1] == workload \
                         and parts[3] == digest:
-                    return float(parts[2])
+                    return float(parts[2]), ("replayed from profiles/dram_traffic.txt (ncu capture of this kernel on this "
+                                             f"workload; source sha256 {digest[:12]} unchanged since)")
     except Exception:
         pass
-    return None
+    return None, "no ncu capture of the kernel as it stands"
 
 
 class ClockSampler:
@@ -124,6 +133,54 @@ def dist_env():
     return rank, local, world
 
 
+def launch_ranks(n: int) -> int:
+    """Start this script again as n ranks of one node (one process per GPU) and return their exit code."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    env = dict(os.environ)
+    # the communicator's own start-up log shows how many ranks joined and which transport they use
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr",
+           "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd, env=env)
+
+
+def init_group(local: int, world: int):
+    """Process group of the ranks torchrun started: NCCL on GPUs (barrier, timing reduction and, for a row-sharded
+    cache, the one all-gather), gloo where there is no GPU (the launcher check only).  Returns the torch device."""
+    import torch
+    import torch.distributed as dist
+    if torch.cuda.is_available():
+        torch.cuda.set_device(local)
+        dev = torch.device("cuda", local)
+        if world > 1 and not dist.is_initialized():
+            dist.init_process_group("nccl", device_id=dev)
+        return dev
+    if world > 1 and not dist.is_initialized():
+        dist.init_process_group("gloo")
+    return torch.device("cpu")
+
+
+def run_launch_check(args):
+    """Starts nothing on the data path: forms the process group, runs the barrier and the max / sum reduction of the
+    timing on made-up numbers (rank r reports r + 1 ms and 10 units), and has rank 0 print what came out."""
+    import torch.distributed as dist
+    from paper_2002_02645_b200 import sharding
+    rank, local, world = dist_env()
+    dev = init_group(local, world)
+    if world > 1:
+        dist.barrier()
+    ms, units = sharding.reduce_timing(float(rank + 1), 10.0, dev)
+    if rank == 0:
+        print(json.dumps({"check": "launch", "n_gpus": world, "requested": args.gpus, "max_ms": ms, "units": units,
+                          "backend": dist.get_backend() if world > 1 else None, "device": dev.type}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ---------------------------------------------------------------------------------------------- workloads
 
 def build_workload(name: str, seed: int, query_seed=None, batch=16):
@@ -178,7 +235,47 @@ def calibrate(cache, calib_dev, percentile):
     return tau
 
 
-def run_ours(args):
+def measure_e2e(args, w, caches, cascade, fence, dev):
+    """The same metric through the host-buffer entry point: pinned host activations copied in, results copied out,
+    every step."""
+    import torch
+    from paper_2002_02645_b200 import binding as fb
+    from paper_2002_02645_b200 import sharding
+    b0 = w.stages[0].queries.shape[0]
+    host_acts = [to_pinned(st.queries) for st in w.stages]
+    h_label = torch.empty(b0, dtype=torch.int32).pin_memory()
+    h_stage = torch.empty(b0, dtype=torch.int32).pin_memory()
+    h_conf = torch.empty(b0, dtype=torch.float32).pin_memory()
+    h_out = fb.LookupOut(b0, w.k, "cpu", with_topk=False)
+    for name in ("label", "conf", "hit"):
+        setattr(h_out, name, getattr(h_out, name).pin_memory())
+
+    def e2e_step():
+        if cascade:
+            fb.cascade_run_host(caches, host_acts, h_label, h_stage, h_conf)
+        else:
+            caches[0].lookup_batch_host(host_acts[0], h_out)
+
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        e2e_step()
+    fence()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    fence()
+    e2e_s = time.perf_counter() - t0
+    e2e_s, e2e_served = sharding.reduce_timing(e2e_s, b0 * e2e_steps, dev)
+    h2d = sum(int(a.numel() * a.element_size()) for a in host_acts)
+    d2h = b0 * 12 if cascade else b0 * 9
+    return {"value": e2e_served / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": 1e3 * e2e_s / e2e_steps}
+
+
+
+def measure_ours(args, workload, batch, *, full=True):
+    """One workload on this rank's GPU; returns the JSON line as a dict (rank 0) or None (other ranks).
+    full=False leaves out the end-to-end leg and the CPU baseline (the "targets" entries of the default run)."""
     import torch
     import torch.distributed as dist
 
@@ -189,10 +286,7 @@ def run_ours(args):
     rank, local, world = dist_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    dev = init_group(local, world)
     if rank == 0:
         fbuild.build_library()
     if world > 1:
@@ -201,8 +295,8 @@ def run_ours(args):
 
     t_gen = time.time()
     # every rank serves its own requests: same caches, batch drawn from the rank's own seed
-    w = build_workload(args.workload, seed=0, query_seed=None if (rank == 0 or args.same_batch) else 1000 + rank,
-                       batch=args.batch)
+    w = build_workload(workload, seed=0, query_seed=None if (rank == 0 or args.same_batch) else 1000 + rank,
+                       batch=batch)
     t_gen = time.time() - t_gen
 
     n_stage = len(w.stages)
@@ -318,7 +412,7 @@ def run_ours(args):
 
     # ---- per-look-up device latency (latency workload): every look-up between its own pair of events
     latency = None
-    if args.workload == "cfg5":
+    if workload == "cfg5":
         n_lat = max(1000, args.steps)
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_lat)]
         fence()
@@ -331,35 +425,9 @@ def run_ours(args):
         latency = {"lookups": n_lat, "p50_us": lat[len(lat) // 2], "p99_us": lat[int(len(lat) * 0.99)],
                    "min_us": lat[0], "max_us": lat[-1]}
 
-    # ---- end to end through the host-buffer entry point
-    host_acts = [to_pinned(st.queries) for st in w.stages]
-    h_label = torch.empty(b0, dtype=torch.int32).pin_memory()
-    h_stage = torch.empty(b0, dtype=torch.int32).pin_memory()
-    h_conf = torch.empty(b0, dtype=torch.float32).pin_memory()
-    h_out = fb.LookupOut(b0, w.k, "cpu", with_topk=False)
-    for name in ("label", "conf", "hit"):
-        setattr(h_out, name, getattr(h_out, name).pin_memory())
-
-    def e2e_step():
-        if cascade:
-            fb.cascade_run_host(caches, host_acts, h_label, h_stage, h_conf)
-        else:
-            caches[0].lookup_batch_host(host_acts[0], h_out)
-
-    e2e_steps = max(3, min(args.steps, 10))
-    for _ in range(2):
-        e2e_step()
-    fence()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        e2e_step()
-    fence()
-    e2e_s = time.perf_counter() - t0
-    e2e_s, e2e_served = sharding.reduce_timing(e2e_s, b0 * e2e_steps, dev)
-    h2d = sum(int(a.numel() * a.element_size()) for a in host_acts)
-    d2h = b0 * 12 if cascade else b0 * 9
-    e2e = {"value": e2e_served / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": 1e3 * e2e_s / e2e_steps}
+    e2e = None
+    if full:
+        e2e = measure_e2e(args, w, caches, cascade, fence, dev)
 
     # ---- roofline of the dominant kernel: the distance kernel of the first (largest) stage
     peaks, peak_src = load_peaks()
@@ -371,7 +439,7 @@ def run_ours(args):
         avg_s = ms0 / n_launch0 * 1e-3
         flops = 2.0 * b0 * n0 * d0
         nbytes = n0 * d0 * st0.cache_vecs.itemsize + b0 * d0 * st0.cache_vecs.itemsize + 4.0 * n0
-        gemm = st0.dtype == "bf16" and b0 > 4
+        gemm = st0.dtype == "bf16" and b0 > 1      # the library's own rule: single requests and fp32 caches stream
         # the events bracket the distance kernel of a look-up: gemm_select_kernel (followed, in wave + tail mode, by
         # its two small tail kernels) or stream_lookup_kernel
         kernel = "gemm_select_kernel" if gemm else "stream_lookup_kernel"
@@ -390,7 +458,8 @@ def run_ours(args):
         # the nominal figures next to the measured ones: 2.25 PFLOP/s dense bf16 and "about 8 TB/s"
         roofline["frac_of_nominal"] = achieved / (2250.0 if tensor_bound else 8000.0)
         roofline["nominal_peak"] = 2250.0 if tensor_bound else 8000.0
-        roofline.update({"traffic": captured_traffic(kernel, w.name), "avg_launch_ms": avg_s * 1e3,
+        traffic, traffic_src = captured_traffic(kernel, w.name)
+        roofline.update({"traffic": traffic, "traffic_source": traffic_src, "avg_launch_ms": avg_s * 1e3,
                          "launches": n_launch0, "algorithmic_flops": flops, "algorithmic_bytes": nbytes})
     stage_info = []
     for l, (ms_l, n_l) in enumerate(prof):
@@ -402,7 +471,7 @@ def run_ours(args):
 
     # ---- the oracle on the host cores, bounded sample (rank 0, single GPU runs only)
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and full and not args.no_cpu_baseline:
         cpu_baseline = time_oracle(w, taus, args.cpu_sample)
 
     if rank == 0:
@@ -423,11 +492,60 @@ def run_ours(args):
             line["ms_per_step_l2_warm"] = ms_warm
         if latency is not None:
             line["latency"] = latency
-        print(json.dumps(line))
+    else:
+        line = None
     for c in caches:
         c.close()
+    del caches, acts, state, out_single
+    torch.cuda.empty_cache()
+    return line
+
+
+def run_ours(args):
+    import torch.distributed as dist
+    rank, _, world = dist_env()
+    line = measure_ours(args, args.workload, args.batch)
+    if rank == 0 and world == 1 and args.workload == "cfg2" and not args.no_targets:
+        line["targets"] = measure_targets(args)
+    if rank == 0:
+        print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def measure_targets(args):
+    """The configurations the two numeric targets sit on, measured in this process after the headline workload:
+    config 3 (largest batch: fraction of the bf16 tensor peak), config 5 at batch 1 / 4 / 16 (fraction of the HBM
+    bandwidth, device-timed latency percentiles over >= 1,000 look-ups) and config 4's per-stage rates.  Every entry
+    carries the clocks sampled during its own timed region."""
+    peaks, peak_src = load_peaks()
+    out = {"peaks": {"source": peak_src, **peaks, "nominal_bf16_tflops": 2250.0, "nominal_hbm_gbs": 8000.0}}
+
+    def brief(line):
+        r = line["roofline"] or {}
+        d = {"workload": line["config"]["workload"], "batch": line["config"]["batch"], "ms_per_step": line["ms_per_step"],
+             "queries_per_s": line["value"], "kernel": r.get("kernel"), "kernel_ms": r.get("avg_launch_ms"),
+             "bound": r.get("bound"), "achieved": r.get("achieved"), "unit": r.get("unit"),
+             "frac_of_measured": r.get("frac"), "frac_of_nominal": r.get("frac_of_nominal"),
+             "clocks": line["clocks"], "gpu_launches": line["gpu_launches"]}
+        if r.get("bound") == "tensor":
+            d["frac_of_measured_sustained"] = r["achieved"] / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+        return d
+
+    l3 = measure_ours(args, "cfg3", 16, full=False)
+    out["config3_batch8192"] = brief(l3)
+    for b in (1, 4, 16):
+        l5 = measure_ours(args, "cfg5", b, full=False)
+        d = brief(l5)
+        d.update({"p50_us": l5["latency"]["p50_us"], "p99_us": l5["latency"]["p99_us"], "lookups_timed": l5["latency"]["lookups"]})
+        out[f"config5_batch{b}"] = d
+    l4 = measure_ours(args, "cfg4", 16, full=False)
+    d = brief(l4)
+    d["arrivals"] = l4["config"]["arrivals"]
+    d["stages"] = [{"stage": s["stage"], "arrivals": s["arrivals"], "distance_kernel_ms": s["distance_kernel_ms"],
+                    "tflops": s["tflops"], "frac_of_measured": s["tflops"] / peaks["bf16_tflops"]} for s in l4["stages"]]
+    out["config4_batch4096"] = d
+    return out
 
 
 # ---------------------------------------------------------------------------------------------- CPU oracle leg
@@ -487,6 +605,7 @@ def run_reference(args):
         else:
             taus.append(float("inf"))
     steps, warmup = max(1, args.steps), max(0, args.warmup)
+    fo.set_threads(len(os.sched_getaffinity(0)))      # a launcher may have set OMP_NUM_THREADS=1 for its ranks
     if args.cpu_sample:
         sample = args.cpu_sample
     else:
@@ -846,14 +965,20 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0", "kmeans", "cfg3-rows", "tau-sweep", "cfg2-proj"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0", "kmeans", "cfg3-rows", "tau-sweep", "cfg2-proj", "launch-check"])
+    ap.add_argument("--no-targets", action="store_true",
+                    help="default workload only: skip the config 3 / 4 / 5 measurements that follow the headline")
     ap.add_argument("--cpu-sample", type=int, default=0,
                     help="requests per oracle timing (0: sized for 10-30 s of CPU work)")
     ap.add_argument("--batch", type=int, default=16, help="batch of the latency workload (cfg5): 1, 4 or 16")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--same-batch", action="store_true", help="every rank serves the same batch")
     args = ap.parse_args()
-    if args.workload == "kmeans":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(launch_ranks(args.gpus))
+    if args.workload == "launch-check":
+        run_launch_check(args)
+    elif args.workload == "kmeans":
         run_kmeans(args)
     elif args.workload == "cfg2-proj" and args.impl == "ours":
         run_projected(args)

@@ -169,7 +169,8 @@ def kmeans_step(points: np.ndarray, centres: np.ndarray, point_labels: np.ndarra
     """One Lloyd iteration plus the tagging of Sec. 2.1 / Sec. 4: assign every point to its nearest centre (squared
     L2, ties to the smaller index), replace each centre by the mean of its points, and record per cluster the most
     frequent model-predicted label (smaller label on ties) with its share."""
-    from paper_2002_02645_b200.datagen import stored_to_f64
+    def stored_to_f64(a):
+        return bf16_bits_to_f64(a) if a.dtype == np.uint16 else np.asarray(a, dtype=np.float64)
     clusters = centres.shape[0]
     r = lookup(points, centres, np.zeros(clusters, np.int32), k=1, tau=0.0)
     assign = r.ni[:, 0].copy()

@@ -95,21 +95,13 @@ int resolve_path(const fi_cache *c, int batch_max) {
     return FI_PATH_GEMM;
 }
 
-fi_status_t ensure_part_scratch(fi_cache *c, size_t entries) {
+// The candidate-list scratch is sized once, at create, for every batch up to max_batch against every cache size up to
+// capacity (gemm_part_entries_bound); a look-up never allocates or synchronises.  A plan that would not fit is a bug of
+// that bound and is refused instead of being run.
+fi_status_t check_part_scratch(const fi_cache *c, size_t entries) {
     if (entries <= c->part_entries) return FI_OK;
-    cudaError_t e = cudaDeviceSynchronize();
-    if (e != cudaSuccess) return cuda_fail(e, "synchronising before growing the look-up scratch");
-    cudaFree(c->part_score);
-    cudaFree(c->part_idx);
-    c->part_score = nullptr;
-    c->part_idx = nullptr;
-    c->part_entries = 0;
-    fi_status_t st = dev_alloc(&c->part_score, entries, "allocating candidate scores");
-    if (st != FI_OK) return st;
-    st = dev_alloc(&c->part_idx, entries, "allocating candidate indices");
-    if (st != FI_OK) return st;
-    c->part_entries = entries;
-    return FI_OK;
+    set_error("look-up scratch too small (%zu entries needed, %zu allocated at create)", entries, c->part_entries);
+    return FI_ERR_CAPACITY;
 }
 
 fi_status_t lookup_impl(fi_cache *c, const void *queries, int64_t ld, const int32_t *row_idx, int32_t batch_max,
@@ -138,7 +130,7 @@ fi_status_t lookup_impl(fi_cache *c, const void *queries, int64_t ld, const int3
             set_error("the tensor-core path needs a bf16 cache");
             return FI_ERR_UNSUPPORTED;
         }
-        st = ensure_part_scratch(c, gemm_part_entries(batch_max, c->size, c->sm_count, c->cfg.k, c->cfg.dim));
+        st = check_part_scratch(c, gemm_part_entries(batch_max, c->size, c->sm_count, c->cfg.k, c->cfg.dim));
         if (st != FI_OK) return st;
         const void *qsrc = queries;
         int64_t qld = ld;
@@ -160,6 +152,31 @@ fi_status_t lookup_impl(fi_cache *c, const void *queries, int64_t ld, const int3
         fa.refine = 1;
     }
     return launch_finalize(c, fa, stream);
+}
+
+// The status words of `n` caches, fetched behind whatever is queued on `stream`; call before the stream is synchronised
+// and hand the words to status_from_words afterwards.
+cudaError_t fetch_status_words(fi_cache *const *caches, int n, int32_t *words, cudaStream_t stream) {
+    cudaError_t e = cudaSuccess;
+    for (int l = 0; l < n && e == cudaSuccess; ++l)
+        e = cudaMemcpyAsync(words + l, caches[l]->status_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, stream);
+    return e;
+}
+
+// FI_ERR_TIMEOUT (and the words cleared) when a kernel of one of the caches gave up on a bounded wait: the results
+// of that call are not to be trusted.
+fi_status_t status_from_words(fi_cache *const *caches, int n, const int32_t *words, const char *who) {
+    fi_status_t st = FI_OK;
+    for (int l = 0; l < n; ++l) {
+        if (words[l] == 0) continue;
+        cudaMemset(caches[l]->status_dev, 0, sizeof(int32_t));
+        if (st == FI_OK) {
+            set_error("%s: a kernel gave up on a bounded wait (code %d, site %d, cache %d); the results are invalid", who,
+                      words[l] & 0xFF, words[l] >> 8, l);
+            st = FI_ERR_TIMEOUT;
+        }
+    }
+    return st;
 }
 
 }  // namespace
@@ -203,6 +220,7 @@ fi_status_t fi_cache_create(const fi_cache_config_t *cfg, fi_cache_t **out) {
     }
     const bool bf16 = cfg->dtype == FI_BF16;
     if ((cfg->dtype != FI_F32 && !bf16) || cfg->dim <= 0 || cfg->dim % (bf16 ? 8 : 4) != 0 || cfg->capacity <= 0 ||
+        cfg->capacity > kMaxEntries ||
         cfg->k < 1 || cfg->k > kMaxK || cfg->max_batch < 1 || cfg->num_classes < 1 ||
         (cfg->rule != FI_HIT_CONF_GT && cfg->rule != FI_HIT_DIST_LE) ||
         (cfg->metric != FI_METRIC_SQL2 && cfg->metric != FI_METRIC_L2) || cfg->path < FI_PATH_AUTO ||
@@ -255,7 +273,7 @@ fi_status_t fi_cache_create(const fi_cache_config_t *cfg, fi_cache_t **out) {
     size_t entries = (size_t)16 * c->sm_count * 4 * cfg->k;
     if (entries < (size_t)cfg->max_batch * cfg->k * 2) entries = (size_t)cfg->max_batch * cfg->k * 2;
     if (bf16) {
-        size_t g = gemm_part_entries(cfg->max_batch, cfg->capacity, c->sm_count, cfg->k, cfg->dim);
+        size_t g = gemm_part_entries_bound(cfg->max_batch, cfg->capacity, c->sm_count, cfg->k, cfg->dim);
         if (g > entries) entries = g;
     }
     if (st == FI_OK) need(dev_alloc(&c->part_score, entries, "allocating candidate scores"));
@@ -276,6 +294,23 @@ fi_status_t fi_cache_create(const fi_cache_config_t *cfg, fi_cache_t **out) {
     if (st == FI_OK) {
         cudaError_t e = cudaMemset(c->status_dev, 0, sizeof(int32_t));
         if (e != cudaSuccess) st = cuda_fail(e, "clearing the status word");
+    }
+    if (st == FI_OK && bf16) {
+        // everything a look-up on the tensor-core path needs is set up here, so that no look-up ever allocates,
+        // synchronises or re-encodes: partial-sum slots (shapes that can reach wave + tail mode), the kernels'
+        // per-device attributes, and tensor maps over all `capacity` rows (rows not yet inserted read as zero and
+        // are masked by the row count the kernels are given)
+        const size_t units = gemm_tail_units(cfg->max_batch, cfg->dim, c->sm_count);
+        if (units > 0) {
+            need(dev_alloc(&c->tail_dump, units * 256 * 256, "allocating the partial-sum buffer of the distance GEMM"));
+            if (st == FI_OK) c->tail_dump_units = units;
+        }
+        if (st == FI_OK) need(prepare_gemm_kernels(cfg->device));
+        if (st == FI_OK) {
+            cudaError_t e = cudaMemset(c->rows, 0, (size_t)cfg->capacity * cfg->dim * c->elem_size);
+            if (e != cudaSuccess) st = cuda_fail(e, "clearing the cache rows");
+        }
+        if (st == FI_OK) need(ensure_tensor_maps(c));
     }
     if (st != FI_OK) {
         free_all(c);
@@ -333,7 +368,6 @@ fi_status_t fi_cache_insert(fi_cache_t *c, const void *vecs, const int32_t *labe
     fi_status_t st = launch_row_norms(dst, c->cfg.dtype, n, c->cfg.dim, c->norms + c->size, stream);
     if (st != FI_OK) return st;
     c->size += n;
-    c->tmaps_ready = false;
     return FI_OK;
 }
 
@@ -367,7 +401,6 @@ fi_status_t fi_cache_clear(fi_cache_t *c) {
         return FI_ERR_INVALID_ARG;
     }
     c->size = 0;
-    c->tmaps_ready = false;
     return FI_OK;
 }
 
@@ -517,10 +550,12 @@ fi_status_t fi_cache_lookup_batch_host(const fi_cache_t *cache, const void *quer
         e = cudaMemcpyAsync(out_host->topk_dist, dev.topk_dist, (size_t)batch * k * 4, cudaMemcpyDeviceToHost, stream);
     if (e == cudaSuccess && out_host->topk_idx)
         e = cudaMemcpyAsync(out_host->topk_idx, dev.topk_idx, (size_t)batch * k * 4, cudaMemcpyDeviceToHost, stream);
+    int32_t word = 0;
+    if (e == cudaSuccess) e = fetch_status_words(&c, 1, &word, stream);
     if (e != cudaSuccess) return cuda_fail(e, "fi_cache_lookup_batch_host: copying results");
     e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return cuda_fail(e, "fi_cache_lookup_batch_host: synchronising");
-    return FI_OK;
+    return status_from_words(&c, 1, &word, "fi_cache_lookup_batch_host");
 }
 
 fi_status_t fi_cascade_run_host(fi_cache_t *const *caches, int32_t num_stages, const void *const *acts_host,
@@ -641,11 +676,13 @@ fi_status_t fi_cascade_run_host(fi_cache_t *const *caches, int32_t num_stages, c
     if (e == cudaSuccess) e = cudaMemcpyAsync(final_conf_host, final_conf, nb * 4, cudaMemcpyDeviceToHost, stream);
     if (e == cudaSuccess && stage_arrivals_host && num_stages > 0)
         e = cudaMemcpyAsync(stage_arrivals_host + 1, counts + 1, (size_t)num_stages * 4, cudaMemcpyDeviceToHost, stream);
+    int32_t words[kMaxHostStages];
+    if (e == cudaSuccess) e = fetch_status_words(caches, num_stages, words, stream);
     if (e != cudaSuccess) return cuda_fail(e, "fi_cascade_run_host: copying results");
     e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return cuda_fail(e, "fi_cascade_run_host: synchronising");
     if (stage_arrivals_host) stage_arrivals_host[0] = batch0;
-    return FI_OK;
+    return status_from_words(caches, num_stages, words, "fi_cascade_run_host");
 }
 
 fi_status_t fi_cache_compute_threshold(fi_cache_t *c, const void *val_acts, int64_t ld_elems, const int32_t *model_labels,
@@ -679,9 +716,15 @@ fi_status_t fi_cache_compute_threshold(fi_cache_t *c, const void *val_acts, int6
         if (st != FI_OK) return st;
     }
     int32_t host[2] = {0, 0};
+    int32_t word = 0;
     e = cudaMemcpyAsync(host, c->calib_acc, sizeof host, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = fetch_status_words(&c, 1, &word, stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return cuda_fail(e, "fi_cache_compute_threshold: reading the result");
+    {
+        const fi_status_t ws = status_from_words(&c, 1, &word, "fi_cache_compute_threshold");
+        if (ws != FI_OK) return ws;   // the cache's threshold is left as it was
+    }
     float tau;
     memcpy(&tau, &host[0], sizeof tau);
     c->cfg.threshold = tau;
@@ -764,8 +807,13 @@ fi_status_t fi_projection_create(int32_t in_dim, int32_t out_dim, int32_t device
     }
     DeviceGuard guard(device);
     const size_t units = product_dump_units(max_batch, out_dim, p->w->sm_count);
-    st = dev_alloc(&p->w->tail_dump, units * 256 * 256, "allocating the projection's partial sums");
-    if (st == FI_OK) p->w->tail_dump_units = units;
+    if (units > p->w->tail_dump_units) {
+        cudaFree(p->w->tail_dump);
+        p->w->tail_dump = nullptr;
+        p->w->tail_dump_units = 0;
+        st = dev_alloc(&p->w->tail_dump, units * 256 * 256, "allocating the projection's partial sums");
+        if (st == FI_OK) p->w->tail_dump_units = units;
+    }
     if (st == FI_OK) st = dev_alloc(&p->zero_labels, (size_t)out_dim, "allocating the projection's labels");
     if (st == FI_OK) st = dev_alloc(&p->zero_bias, (size_t)out_dim, "allocating the projection's zero bias");
     unsigned char *y = nullptr;

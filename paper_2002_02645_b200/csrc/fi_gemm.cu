@@ -25,6 +25,8 @@
 // Every wait is bounded: a wait that runs out sets the cache's status word and the CTA drains and returns.
 #include <cuda_bf16.h>
 
+#include <mutex>
+
 #include "fi_internal.cuh"
 
 namespace fi {
@@ -1018,13 +1020,7 @@ fi_status_t prepare_gemm_kernel(Kern kern, const char *what) {
 template <int KP, int MSUB>
 fi_status_t launch_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, const int32_t *count_dev, bool tail_possible,
                       cudaStream_t stream) {
-    static bool attr_set = false;
-    auto kern = gemm_select_kernel<KP, MSUB>;
-    if (!attr_set) {
-        const fi_status_t ps = prepare_gemm_kernel(kern, "distance GEMM");
-        if (ps != FI_OK) return ps;
-        attr_set = true;
-    }
+    auto kern = gemm_select_kernel<KP, MSUB>;   // prepared for this device by prepare_gemm_kernels (fi_cache_create)
     // every bound starts at a huge finite value (0x7F7F7F7F as a float is 3.4e38)
     if (cudaMemsetAsync(c->row_bound, 0x7F, ((size_t)batch_max + 256) * KP * sizeof(int32_t), stream) != cudaSuccess) {
         set_error("cannot reset the row bounds");
@@ -1074,14 +1070,43 @@ fi_status_t launch_wait_selftest(fi_cache *c, long long limit_cycles, cudaStream
     return check_launch("wait_selftest_kernel");
 }
 
+// The maps cover all `capacity` rows and are encoded once, at create: the kernels are told how many rows count
+// (columns past that number get an infinite score), so appending entries never touches the maps.
 fi_status_t ensure_tensor_maps(fi_cache *c) {
     if (c->tmaps_ready) return FI_OK;
-    fi_status_t st = encode_bf16_map(&c->tmap_rows64, c->rows, (uint64_t)c->size, (uint64_t)c->cfg.dim, (uint64_t)c->cfg.dim, 64);
+    fi_status_t st = encode_bf16_map(&c->tmap_rows64, c->rows, (uint64_t)c->cfg.capacity, (uint64_t)c->cfg.dim, (uint64_t)c->cfg.dim, 64);
     if (st != FI_OK) return st;
-    st = encode_bf16_map(&c->tmap_rows16, c->rows, (uint64_t)c->size, (uint64_t)c->cfg.dim, (uint64_t)c->cfg.dim, 16);
+    st = encode_bf16_map(&c->tmap_rows16, c->rows, (uint64_t)c->cfg.capacity, (uint64_t)c->cfg.dim, (uint64_t)c->cfg.dim, 16);
     if (st != FI_OK) return st;
     c->tmaps_ready = true;
     return FI_OK;
+}
+
+// Every instantiation of the distance GEMM is prepared once per device (the shared-memory reservation is a
+// per-device attribute), under a lock, before the first cache on that device can launch one.
+fi_status_t prepare_gemm_kernels(int device) {
+    static std::mutex mu;
+    static bool done[kMaxDevices] = {};
+    if (device < 0 || device >= kMaxDevices) {
+        set_error("device ordinal %d outside 0..%d", device, kMaxDevices - 1);
+        return FI_ERR_INVALID_ARG;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    if (done[device]) return FI_OK;
+    fi_status_t st = FI_OK;
+    auto prep = [&](auto kern) {
+        if (st == FI_OK) st = prepare_gemm_kernel(kern, "distance GEMM");
+    };
+    prep(gemm_select_kernel<4, 1>);
+    prep(gemm_select_kernel<8, 1>);
+    prep(gemm_select_kernel<16, 1>);
+    prep(gemm_select_kernel<32, 1>);
+    prep(gemm_select_kernel<4, 2>);
+    prep(gemm_select_kernel<8, 2>);
+    prep(gemm_select_kernel<16, 2>);
+    prep(gemm_select_kernel<32, 2>);
+    if (st == FI_OK) done[device] = true;
+    return st;
 }
 
 size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, int dim) {
@@ -1095,6 +1120,34 @@ size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, i
         if (e > worst) worst = e;
     }
     return worst;
+}
+
+size_t gemm_part_entries_bound(int max_batch, int64_t capacity, int sm_count, int k, int dim) {
+    // lists per query: at most one per range (ranges <= CTAs, and <= 16-row blocks of the cache), times two for
+    // 128-row tiles (two epilogue warps per row); wave + tail mode has one list per 256-row tile of the cache,
+    // at most 1.5 x CTAs of them
+    const size_t n16 = (size_t)((capacity + 15) / 16);
+    const size_t list_len = (size_t)gemm_list_len(k);
+    auto entries = [&](int rows, int tile_m) {
+        const size_t f = tile_m == kTileM ? 2 : 1;
+        size_t lists = (size_t)sm_count * f;
+        if (tile_m != kTileM && lists < (size_t)sm_count + sm_count / 2) lists = (size_t)sm_count + sm_count / 2;
+        if (lists > n16 * f) lists = n16 * f;
+        if (lists < f) lists = f;
+        const size_t padded = (size_t)((rows + tile_m - 1) / tile_m) * tile_m;
+        return padded * lists * list_len;
+    };
+    size_t worst = entries(max_batch < kTileM ? max_batch : (gemm_tile_m(max_batch, dim) == kTileM ? max_batch : kTileM), kTileM);
+    if (gemm_tile_m(max_batch, dim) != kTileM) {
+        const size_t e = entries(max_batch, 2 * kTileM);
+        if (e > worst) worst = e;
+    }
+    return worst;
+}
+
+size_t gemm_tail_units(int max_batch, int dim, int sm_count) {
+    const int num_kb = (dim + kBlockK - 1) / kBlockK;
+    return gemm_tile_m(max_batch, dim) == 2 * kTileM && num_kb >= 64 ? (size_t)sm_count : 0;
 }
 
 // Can a batch of at most batch_max requests against the current cache end up in wave + tail mode?
@@ -1125,20 +1178,9 @@ fi_status_t launch_gemm_select(fi_cache *c, const void *queries_compact, int64_t
     if (st != FI_OK) return st;
     const bool tail_possible = tail_mode_possible(c, batch_max);
     if (tail_possible && c->tail_dump_units < (size_t)c->sm_count) {
-        // one slot of 256 x 256 partial sums per CTA; allocated the first time a shape can need it
-        cudaError_t e = cudaStreamSynchronize(stream);
-        if (e == cudaSuccess) {
-            cudaFree(c->tail_dump);
-            c->tail_dump = nullptr;
-            c->tail_dump_units = 0;
-            e = cudaMalloc(reinterpret_cast<void **>(&c->tail_dump), (size_t)c->sm_count * kMaxTileN * 2 * kTileM * sizeof(float));
-        }
-        if (e != cudaSuccess) {
-            set_error("cannot allocate the partial-sum buffer of the distance GEMM: %s", cudaGetErrorString(e));
-            cudaGetLastError();
-            return e == cudaErrorMemoryAllocation ? FI_ERR_OOM : FI_ERR_CUDA;
-        }
-        c->tail_dump_units = (size_t)c->sm_count;
+        // one slot of 256 x 256 partial sums per CTA, allocated at create for every cache whose shapes can get here
+        set_error("the distance GEMM's partial-sum buffer is missing (%zu slots, %d needed)", c->tail_dump_units, c->sm_count);
+        return FI_ERR_CAPACITY;
     }
     if (gemm_tile_m(batch_max, c->cfg.dim) == kTileM) return launch_msub<1>(c, tq, batch_max, count_dev, false, stream);
     return launch_msub<2>(c, tq, batch_max, count_dev, tail_possible, stream);
@@ -1168,13 +1210,7 @@ fi_status_t launch_gemm_project(fi_cache *w, const void *queries_compact, int64_
     CUtensorMap tq;
     st = encode_bf16_map(&tq, queries_compact, (uint64_t)batch_max, (uint64_t)w->cfg.dim, (uint64_t)ld_elems, kTileM);
     if (st != FI_OK) return st;
-    static bool attr_set = false;
-    auto kern = gemm_select_kernel<8, 2>;
-    if (!attr_set) {
-        const fi_status_t ps = prepare_gemm_kernel(kern, "projection GEMM");
-        if (ps != FI_OK) return ps;
-        attr_set = true;
-    }
+    auto kern = gemm_select_kernel<8, 2>;   // prepared for this device when the weights' cache object was created
     kern<<<w->sm_count, kGemmThreads, kGemmSmemBytes, stream>>>(tq, w->tmap_rows64, w->tmap_rows16, w->norms,
                                                                (long long)w->size, w->cfg.dim, batch_max, count_dev, 1,
                                                                w->part_score, w->part_idx, w->plan_dev, w->row_bound,

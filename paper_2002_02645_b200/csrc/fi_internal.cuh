@@ -10,9 +10,11 @@
 namespace fi {
 
 constexpr int kMaxK = 32;          // largest k of a look-up
+constexpr long long kMaxEntries = 2147483647ll - 255;   // cache entries are indexed with int32 (tiles may overshoot by < 256)
 constexpr int kStreamMaxBatch = 1; // batches up to this size take the streaming kernel under FI_PATH_AUTO (bf16)
 constexpr int kTileM = 128;        // queries per MMA (= TMEM lanes); a CTA tile holds 128 or 256 queries
 constexpr int kMaxHostStages = 64; // stages a host-driven cascade may have
+constexpr int kMaxDevices = 64;    // device ordinals the per-device set-up tables cover
 constexpr int kProfSlots = 256;    // look-ups whose distance-kernel time is kept
 
 // Candidates kept per query by the GEMM path before the exact re-ranking: k plus a margin of 3,
@@ -266,6 +268,12 @@ size_t product_dump_units(int max_batch, int64_t n_rows, int sm_count);
 fi_status_t launch_wait_selftest(fi_cache *c, long long limit_cycles, cudaStream_t stream);
 fi_status_t ensure_tensor_maps(fi_cache *c);
 size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, int dim);
+// upper bound of gemm_part_entries over every batch <= max_batch and every cache size <= capacity
+size_t gemm_part_entries_bound(int max_batch, int64_t capacity, int sm_count, int k, int dim);
+// slots of 256 x 256 partial sums a cache's look-ups can need (wave + tail mode), 0 when that mode cannot occur
+size_t gemm_tail_units(int max_batch, int dim, int sm_count);
+// one-time, per-device set-up of every instantiation of the distance GEMM (shared-memory reservation, register check)
+fi_status_t prepare_gemm_kernels(int device);
 int gemm_tile_m(int batch_max, int dim);
 
 }  // namespace fi

@@ -16,7 +16,6 @@ namespace {
 constexpr int kNoAllocMaxBatch = 256;
 constexpr size_t kNoAllocEntries = (size_t)kNoAllocMaxBatch * kMaxK * 64;   // 524,288 (score, index) pairs
 constexpr size_t kNoAllocBytes = kNoAllocEntries * 8;                       // 4 MiB
-constexpr int kMaxDevices = 64;
 
 // scratch of the streaming look-up: candidate scores, then candidate indices
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
@@ -74,6 +73,11 @@ extern "C" fi_status_t fi_lookup_noalloc(const void *cache_vecs, const int32_t *
     if ((dtype != FI_F32 && !bf16) || dim <= 0 || dim % (bf16 ? 8 : 4) != 0 || k < 1 || k > kMaxK ||
         (rule != FI_HIT_CONF_GT && rule != FI_HIT_DIST_LE) || (metric != FI_METRIC_SQL2 && metric != FI_METRIC_L2)) {
         set_error("fi_lookup_noalloc: invalid dtype, dim, k, rule or metric");
+        return FI_ERR_INVALID_ARG;
+    }
+    if (n_entries > kMaxEntries) {
+        set_error("fi_lookup_noalloc: %lld entries exceed the int32 index range (at most %lld)", (long long)n_entries,
+                  (long long)kMaxEntries);
         return FI_ERR_INVALID_ARG;
     }
     if (batch > kNoAllocMaxBatch) {

@@ -108,3 +108,32 @@ def test_row_sharding_two_ranks_gloo(tmp_path):
     port = _free_port()
     mp.spawn(_row_shard_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
     assert (tmp_path / "result0").read_text() == "ok" and (tmp_path / "result1").read_text() == "ok"
+
+
+def _bench(*argv, timeout=600):
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    proc = subprocess.run([sys.executable, os.path.join(root, "bench.py"), *argv], stdout=subprocess.PIPE,
+                          stderr=subprocess.PIPE, text=True, timeout=timeout, env=env, cwd=root)
+    assert proc.returncode == 0, proc.stderr[-2000:]
+    lines = [l for l in proc.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, proc.stdout          # rank 0 alone prints, and exactly one line
+    return json.loads(lines[0])
+
+
+def test_bench_gpus_flag_starts_that_many_ranks():
+    """`bench.py --gpus 2` without a launcher around it starts two ranks itself; they form a process group (gloo here,
+    NCCL on GPUs), meet at the barrier, and the timing reduction takes the slowest rank's time and everybody's work."""
+    line = _bench("--gpus", "2", "--workload", "launch-check")
+    assert line["n_gpus"] == 2 and line["requested"] == 2
+    assert line["max_ms"] == 2.0 and line["units"] == 20.0 and line["backend"] == "gloo"
+
+
+def test_bench_reference_arm_under_two_ranks_prints_one_line():
+    line = _bench("--gpus", "2", "--impl", "reference", "--workload", "cfg2-small", "--steps", "1", "--warmup", "0",
+                  "--cpu-sample", "2")
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
