@@ -290,6 +290,28 @@ fi_status_t fi_cache_selftest_wait(fi_cache_t *cache, int64_t limit_cycles, void
 fi_status_t fi_cache_poll_status(fi_cache_t *cache);
 
 /*
+ * Certificate of the tensor-core path (bf16 caches, batches of 2 and more; the paper has no counterpart: it looks up
+ * with exact distances on the CPU).  The distance GEMM ranks cache rows by a score accumulated in fp32 on the tensor
+ * cores and hands a short candidate list per request to the exact re-ranking.  With E = eps (||q||^2 + max ||c||^2),
+ * eps = (dim / 16 + 4) * 2^-23, taken as the bound of a score's error (one dropped unit in the last place per
+ * accumulation step of 16 columns), a request is CERTIFIED when the k-th exact
+ * distance among its candidates is below (largest candidate score) + ||q||^2 - E: then no cache row outside the list
+ * can be one of the k nearest, and the neighbours returned are the exact ones.  Look-ups on the streaming path use
+ * exact distances throughout and are always certified.
+ *   fi_cache_read_certificate: synchronises the device; returns and clears (nullable pointers are skipped) how many
+ *     requests since the last read had no certificate, how many of those the repair pass did not look up again, and
+ *     the largest score error observed on candidates, relative to ||q||^2 + max ||c||^2 (compare with eps).
+ *   fi_cache_read_slot_certificates: synchronises; copies the flags of the cache's most recent look-up (1 = certified or
+ *     repaired) for slots 0..n-1 to host memory.
+ *   fi_cache_set_repair: with repair on, every look-up on the tensor-core path is followed by a second pass in which
+ *     the streaming kernel looks the uncertified requests up again with exact distances (at most 64 per look-up; the
+ *     list stays on the device, and the two extra kernels return at once when it is empty).  Off by default.
+ */
+fi_status_t fi_cache_set_repair(fi_cache_t *cache, int32_t enable);
+fi_status_t fi_cache_read_certificate(fi_cache_t *cache, int64_t *uncertified, int64_t *unrepaired, float *max_score_error);
+fi_status_t fi_cache_read_slot_certificates(fi_cache_t *cache, uint8_t *flags_host, int32_t n);
+
+/*
  * Device timing of the distance kernel (the tensor-core GEMM or the streaming kernel) of later look-ups on
  * this cache: with profiling on, each look-up records a CUDA event before and after that kernel on the
  * caller's stream (up to 256 look-ups are kept; older ones are overwritten).  fi_cache_read_profile

@@ -27,7 +27,8 @@ EXPORTS = ["fi_cache_create", "fi_cache_destroy", "fi_cache_insert", "fi_cache_s
            "fi_cache_read_profile", "fi_lookup_noalloc", "fi_cache_compute_threshold", "fi_cache_clear", "fi_kmeans_step", "fi_cache_selftest_wait", "fi_cache_neighbor_tuples", "fi_merge_shard_lookups",
            "fi_projection_create", "fi_projection_destroy", "fi_projection_set_weights", "fi_projection_apply", "fi_projection_poll_status", "fi_projection_set_profiling",
            "fi_projection_read_profile",
-           "fi_cascade_step_projected", "fi_launch_count", "fi_last_error", "fi_status_string"]
+           "fi_cascade_step_projected", "fi_cache_set_repair", "fi_cache_read_certificate",
+           "fi_cache_read_slot_certificates", "fi_launch_count", "fi_last_error", "fi_status_string"]
 
 
 class fi_cache_config_t(ctypes.Structure):
@@ -98,6 +99,9 @@ def load_library(path: Optional[str] = None):
                                                ctypes.POINTER(i64), vp]
     lib.fi_lookup_noalloc.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, i32, ctypes.c_float, vp, i64, i32,
                                       ctypes.POINTER(fi_lookup_out_t), vp]
+    lib.fi_cache_set_repair.argtypes = [vp, i32]
+    lib.fi_cache_read_certificate.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(ctypes.c_float)]
+    lib.fi_cache_read_slot_certificates.argtypes = [vp, vp, i32]
     lib.fi_cache_set_profiling.argtypes = [vp, i32]
     lib.fi_cache_read_profile.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.fi_launch_count.argtypes = []
@@ -219,6 +223,22 @@ class FreezeCache:
 
     def poll_status(self) -> None:
         _check(self._lib.fi_cache_poll_status(self._h))
+
+    # -- fi_cache_set_repair / fi_cache_read_certificate / fi_cache_read_slot_certificates
+    def set_repair(self, enable: bool) -> None:
+        _check(self._lib.fi_cache_set_repair(self._h, 1 if enable else 0))
+
+    def read_certificate(self):
+        """(requests without a certificate since the last read, of those not repaired, largest observed score error)."""
+        unc, unrep, err = ctypes.c_int64(0), ctypes.c_int64(0), ctypes.c_float(0.0)
+        _check(self._lib.fi_cache_read_certificate(self._h, ctypes.byref(unc), ctypes.byref(unrep), ctypes.byref(err)))
+        return int(unc.value), int(unrep.value), float(err.value)
+
+    def slot_certificates(self, n: int) -> torch.Tensor:
+        """Flags of the most recent look-up, slots 0..n-1 (host uint8 tensor, 1 = certified or repaired)."""
+        flags = torch.zeros(max(n, 1), dtype=torch.uint8)
+        _check(self._lib.fi_cache_read_slot_certificates(self._h, flags.data_ptr(), int(n)))
+        return flags[:n]
 
     # -- fi_cache_neighbor_tuples
     def neighbor_tuples(self, topk_idx: torch.Tensor, index_offset: int):

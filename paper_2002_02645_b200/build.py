@@ -7,7 +7,8 @@ import sys
 
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
-LIB = os.path.join(PKG, "libficache.so")
+# FICACHE_LIB names another build of the library to load instead of the in-tree one (it is then never rebuilt here)
+LIB = os.environ.get("FICACHE_LIB") or os.path.join(PKG, "libficache.so")
 SOURCES = ["fi_api.cu", "fi_stream.cu", "fi_finalize.cu", "fi_gemm.cu", "fi_noalloc.cu", "fi_kmeans.cu"]
 HEADERS = [os.path.join(CSRC, "fi_internal.cuh"), os.path.join(os.path.dirname(PKG), "include", "fi.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -33,6 +34,8 @@ def stale() -> bool:
 def build_library(force: bool = False, verbose: bool = False) -> str:
     """Compile csrc/*.cu into libficache.so next to this file; returns its path.  The sources are compiled side by
     side into objects under _build/ (only those older than their source or a header) and then linked."""
+    if os.environ.get("FICACHE_LIB"):
+        return LIB
     if not force and not stale():
         return LIB
     from concurrent.futures import ThreadPoolExecutor

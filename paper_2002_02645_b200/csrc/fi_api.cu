@@ -64,6 +64,9 @@ void free_all(fi_cache *c) {
     cudaFree(c->km_dist);
     cudaFree(c->km_partial);
     cudaFree(c->status_dev);
+    cudaFree(c->cert_dev);
+    cudaFree(c->slot_cert);
+    cudaFree(c->repair_list);
     cudaFree(c->h2d_stage);
     if (c->copy_ev) {
         for (int i = 0; i < kMaxHostStages; ++i) cudaEventDestroy(c->copy_ev[i]);
@@ -115,6 +118,8 @@ fi_status_t lookup_impl(fi_cache *c, const void *queries, int64_t ld, const int3
     fa.batch_max = batch_max;
     fa.count_dev = count_dev;
     fa.out = out;
+    fa.out_slot = nullptr;
+    fa.fill_repair_list = false;
     fi_status_t st;
     if (path == FI_PATH_STREAM) {
         int parts = 1;
@@ -150,6 +155,30 @@ fi_status_t lookup_impl(fi_cache *c, const void *queries, int64_t ld, const int3
         fa.parts = -1;
         fa.list_len = -1;
         fa.refine = 1;
+        if (c->repair_on) {
+            // Exact repair: queries whose neighbours the certificate cannot prove are looked up again by the streaming
+            // kernel (direct fp32 distances over the whole cache).  The list and its length stay on the device; the
+            // kernels of the second pass return at once when the list is empty.
+            fa.fill_repair_list = true;
+            cudaError_t e = cudaMemsetAsync(c->cert_dev + 2, 0, sizeof(int32_t), stream);
+            if (e != cudaSuccess) return cuda_fail(e, "clearing the repair list");
+            st = launch_finalize(c, fa, stream);
+            if (st != FI_OK) return st;
+            int parts = 1;
+            // the queries the distance GEMM read are indexed by slot (gathered copy, or the caller's rows as they are)
+            st = launch_stream_lookup(c, fa.queries, fa.ld_elems, c->repair_list, kRepairCap, c->cert_dev + 2, &parts, stream);
+            if (st != FI_OK) return st;
+            FinalizeArgs fr = fa;
+            fr.row_idx = nullptr;
+            fr.batch_max = kRepairCap;
+            fr.count_dev = c->cert_dev + 2;
+            fr.parts = parts;
+            fr.list_len = c->cfg.k;
+            fr.refine = 0;
+            fr.out_slot = c->repair_list;
+            fr.fill_repair_list = false;
+            return launch_finalize(c, fr, stream);
+        }
     }
     return launch_finalize(c, fa, stream);
 }
@@ -291,6 +320,14 @@ fi_status_t fi_cache_create(const fi_cache_config_t *cfg, fi_cache_t **out) {
     if (st == FI_OK && bf16)
         need(dev_alloc(&c->row_bound, ((size_t)cfg->max_batch + 256) * gemm_list_len(cfg->k), "allocating the row bounds"));
     if (st == FI_OK) need(dev_alloc(&c->status_dev, 1, "allocating the status word"));
+    if (st == FI_OK) need(dev_alloc(&c->cert_dev, (size_t)kCertWords, "allocating the certificate block"));
+    if (st == FI_OK) need(dev_alloc(&c->slot_cert, (size_t)cfg->max_batch, "allocating the certificate flags"));
+    if (st == FI_OK) need(dev_alloc(&c->repair_list, (size_t)kRepairCap, "allocating the repair list"));
+    if (st == FI_OK) {
+        cudaError_t e = cudaMemset(c->cert_dev, 0, kCertWords * sizeof(int32_t));
+        if (e == cudaSuccess) e = cudaMemset(c->slot_cert, 1, (size_t)cfg->max_batch);
+        if (e != cudaSuccess) st = cuda_fail(e, "clearing the certificate block");
+    }
     if (st == FI_OK) {
         cudaError_t e = cudaMemset(c->status_dev, 0, sizeof(int32_t));
         if (e != cudaSuccess) st = cuda_fail(e, "clearing the status word");
@@ -365,7 +402,7 @@ fi_status_t fi_cache_insert(fi_cache_t *c, const void *vecs, const int32_t *labe
         fi_status_t st = check_launch("fill_f32_kernel");
         if (st != FI_OK) return st;
     }
-    fi_status_t st = launch_row_norms(dst, c->cfg.dtype, n, c->cfg.dim, c->norms + c->size, stream);
+    fi_status_t st = launch_row_norms(dst, c->cfg.dtype, n, c->cfg.dim, c->norms + c->size, c->cert_dev + 3, stream);
     if (st != FI_OK) return st;
     c->size += n;
     return FI_OK;
@@ -401,6 +438,8 @@ fi_status_t fi_cache_clear(fi_cache_t *c) {
         return FI_ERR_INVALID_ARG;
     }
     c->size = 0;
+    DeviceGuard guard(c->cfg.device);
+    cudaMemsetAsync(c->cert_dev + 3, 0, sizeof(int32_t), nullptr);   // largest norm of the entries held: none now
     return FI_OK;
 }
 
@@ -1009,6 +1048,46 @@ fi_status_t fi_cache_read_profile(fi_cache_t *c, float *total_ms, int32_t *launc
     }
     *launches = n;
     c->prof_n = 0;
+    return FI_OK;
+}
+
+fi_status_t fi_cache_set_repair(fi_cache_t *c, int32_t enable) {
+    if (!c) {
+        set_error("fi_cache_set_repair: null cache");
+        return FI_ERR_INVALID_ARG;
+    }
+    c->repair_on = enable != 0;
+    return FI_OK;
+}
+
+fi_status_t fi_cache_read_certificate(fi_cache_t *c, int64_t *uncertified, int64_t *unrepaired, float *max_score_error) {
+    if (!c) {
+        set_error("fi_cache_read_certificate: null cache");
+        return FI_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(c->cfg.device);
+    cudaError_t e = cudaDeviceSynchronize();
+    int32_t w[kCertWords] = {0, 0, 0, 0, 0};
+    if (e == cudaSuccess) e = cudaMemcpy(w, c->cert_dev, sizeof w, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaMemset(c->cert_dev, 0, 2 * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(c->cert_dev + 4, 0, sizeof(int32_t));
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cache_read_certificate");
+    if (uncertified) *uncertified = w[0];
+    if (unrepaired) *unrepaired = w[4];
+    if (max_score_error) memcpy(max_score_error, &w[1], sizeof(float));
+    return FI_OK;
+}
+
+fi_status_t fi_cache_read_slot_certificates(fi_cache_t *c, uint8_t *flags_host, int32_t n) {
+    if (!c || n < 0 || n > c->cfg.max_batch || (n > 0 && !flags_host)) {
+        set_error("fi_cache_read_slot_certificates: null argument or more slots than max_batch");
+        return FI_ERR_INVALID_ARG;
+    }
+    if (n == 0) return FI_OK;
+    DeviceGuard guard(c->cfg.device);
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(flags_host, c->slot_cert, (size_t)n, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cache_read_slot_certificates");
     return FI_OK;
 }
 

@@ -52,6 +52,15 @@ struct FinalizeParams {
     uint8_t *out_hit;
     float *out_topk_dist;
     int32_t *out_topk_idx;
+    // certificate of the tensor-core path (refine = 1): is every cache row outside the candidate list provably farther
+    // than the k-th neighbour?  eps bounds the relative error of a score against ||q||^2 + max ||c||^2.
+    float eps;
+    int32_t *cert;            // [0] queries without a certificate, [1] largest observed score error (float bits, relative
+                              // to ||q||^2 + max ||c||^2), [2] length of the repair list, [3] max ||c||^2 (float bits)
+    uint8_t *slot_cert;       // [batch] 1 = certified
+    int32_t *repair_list;     // slots to look up again with exact distances (nullable: no repair)
+    int repair_cap;
+    const int32_t *out_slot;  // nullable: result b goes to output slot out_slot[b] (the repair pass)
 };
 
 __device__ __forceinline__ uint4 ld16(const void *p) {
@@ -87,6 +96,37 @@ __device__ __forceinline__ float sqdiff16<uint16_t>(uint4 q, uint4 x, float acc)
     return acc;
 }
 
+template <typename T>
+__device__ __forceinline__ float sqnorm16(uint4 q, float acc);
+template <>
+__device__ __forceinline__ float sqnorm16<float>(uint4 q, float acc) {
+    acc = fmaf(__uint_as_float(q.x), __uint_as_float(q.x), acc);
+    acc = fmaf(__uint_as_float(q.y), __uint_as_float(q.y), acc);
+    acc = fmaf(__uint_as_float(q.z), __uint_as_float(q.z), acc);
+    return fmaf(__uint_as_float(q.w), __uint_as_float(q.w), acc);
+}
+template <>
+__device__ __forceinline__ float sqnorm16<uint16_t>(uint4 q, float acc) {
+    uint32_t qw[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float a = __uint_as_float(qw[i] << 16), b = __uint_as_float(qw[i] & 0xFFFF0000u);
+        acc = fmaf(a, a, acc);
+        acc = fmaf(b, b, acc);
+    }
+    return acc;
+}
+
+// Certificate of one query on the tensor-core path.  The distance kernel ranks cache rows by an approximate score
+// s^ = ||c||^2 - 2 q.c (bf16 products accumulated in fp32), whose error against the true s = d - ||q||^2 is taken
+// to be at most E = eps (||q||^2 + max ||c||^2).  Its candidate list holds the `want` smallest scores, so every row
+// outside the list has s^ >= s_last, hence a true distance >= s_last + ||q||^2 - E.  If the k-th exact distance found
+// among the candidates is below that, no row outside the list can be among the k nearest: the neighbours are proven
+// to be the exact ones.  (A list with fewer than `want` entries holds every row that counts.)
+__device__ __forceinline__ bool certified(float d_k, float s_last, float qq, float c_max, float eps, bool list_full) {
+    return !list_full || d_k < s_last + qq - eps * (qq + c_max);
+}
+
 __device__ __forceinline__ bool pair_less(float s, int i, float t, int j) { return s < t || (s == t && i < j); }
 
 // One query, finished by all threads of a CTA together.
@@ -99,6 +139,7 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
     __shared__ float cand_w[kMaxK];
     __shared__ int32_t red_k[kFinWarps];
     __shared__ int32_t red_i[kFinWarps];
+    __shared__ float qq_sh;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int entries = parts * list_len;
@@ -206,7 +247,8 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
         const int chunks = p.dim / (16 / (int)sizeof(T));
         for (int j = warp; j < cand_n; j += kFinWarps) {
             const T *x = reinterpret_cast<const T *>(p.X) + (int64_t)cand_i[j] * p.dim;
-            float a0 = 0.f, a1 = 0.f;
+            float a0 = 0.f, a1 = 0.f, n0 = 0.f, n1 = 0.f;
+            const bool with_norm = j == 0;   // ||q||^2 for the certificate rides along with the first candidate
             int c = lane;
             for (; c + 32 < chunks; c += 64) {
                 uint4 x0 = ld16(reinterpret_cast<const uint4 *>(x) + c);
@@ -215,13 +257,26 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
                 uint4 q1 = ld16(reinterpret_cast<const uint4 *>(q) + c + 32);
                 a0 = sqdiff16<T>(q0, x0, a0);
                 a1 = sqdiff16<T>(q1, x1, a1);
+                if (with_norm) {
+                    n0 = sqnorm16<T>(q0, n0);
+                    n1 = sqnorm16<T>(q1, n1);
+                }
             }
-            for (; c < chunks; c += 32)
-                a0 = sqdiff16<T>(ld16(reinterpret_cast<const uint4 *>(q) + c), ld16(reinterpret_cast<const uint4 *>(x) + c), a0);
-            float a = a0 + a1;
+            for (; c < chunks; c += 32) {
+                const uint4 q0 = ld16(reinterpret_cast<const uint4 *>(q) + c);
+                a0 = sqdiff16<T>(q0, ld16(reinterpret_cast<const uint4 *>(x) + c), a0);
+                if (with_norm) n0 = sqnorm16<T>(q0, n0);
+            }
+            float a = a0 + a1, nq = n0 + n1;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
-            if (lane == 0) cand_d[j] = a;
+            for (int o = 16; o > 0; o >>= 1) {
+                a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
+                nq += __shfl_xor_sync(0xFFFFFFFFu, nq, o);
+            }
+            if (lane == 0) {
+                cand_d[j] = a;
+                if (with_norm) qq_sh = nq;
+            }
         }
     } else {
         if (tid < cand_n) cand_d[tid] = cand_s[tid];
@@ -230,6 +285,17 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
 
     // ---- order by (distance, index), vote, hit
     if (tid == 0) {
+        const int o = p.out_slot ? p.out_slot[b] : b;
+        // the certificate needs the scores as the merge left them (cand_s keeps that order; the sort below moves only
+        // distances, indices, labels and weights)
+        float s_last = 0.f, err_max = 0.f;
+        const float c_max = p.cert ? __int_as_float(p.cert[3]) : 0.f;
+        if (p.refine && p.cert && cand_n > 0) {
+            s_last = cand_s[cand_n - 1];
+            const float denom = qq_sh + c_max;
+            for (int a = 0; a < cand_n; ++a) err_max = fmaxf(err_max, fabsf(cand_s[a] + qq_sh - cand_d[a]));
+            err_max = denom > 0.f ? err_max / denom : 0.f;
+        }
         for (int a = 1; a < cand_n; ++a) {
             const float d = cand_d[a], w = cand_w[a];
             const int i = cand_i[a], l = cand_lab[a];
@@ -273,13 +339,31 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
             }
         }
         bool hit = k_eff > 0 && (p.rule == FI_HIT_CONF_GT ? best_c > p.tau : best_dwin <= p.tau);
-        p.out_label[b] = best_label;
-        p.out_conf[b] = best_c;
-        p.out_hit[b] = hit ? 1 : 0;
+        p.out_label[o] = best_label;
+        p.out_conf[o] = best_c;
+        p.out_hit[o] = hit ? 1 : 0;
         if (p.out_topk_dist)
-            for (int j = 0; j < p.k; ++j) p.out_topk_dist[(int64_t)b * p.k + j] = j < k_eff ? cand_d[j] : kInf;
+            for (int j = 0; j < p.k; ++j) p.out_topk_dist[(int64_t)o * p.k + j] = j < k_eff ? cand_d[j] : kInf;
         if (p.out_topk_idx)
-            for (int j = 0; j < p.k; ++j) p.out_topk_idx[(int64_t)b * p.k + j] = j < k_eff ? cand_i[j] : -1;
+            for (int j = 0; j < p.k; ++j) p.out_topk_idx[(int64_t)o * p.k + j] = j < k_eff ? cand_i[j] : -1;
+        if (p.cert && p.slot_cert) {
+            bool ok = true;   // exact distances throughout (streaming lists, the repair pass): nothing to certify
+            if (p.refine && k_eff > 0) {
+                ok = certified(cand_d[k_eff - 1], s_last, qq_sh, c_max, p.eps, cand_n >= want);
+                if (err_max > 0.f) atomicMax(p.cert + 1, __float_as_int(err_max));
+            }
+            p.slot_cert[o] = ok ? 1 : 0;
+            if (!ok) {
+                atomicAdd(p.cert, 1);
+                if (p.repair_list) {
+                    const int pos = atomicAdd(p.cert + 2, 1);
+                    if (pos < p.repair_cap) p.repair_list[pos] = b;
+                    else atomicAdd(p.cert + 4, 1);
+                } else {
+                    atomicAdd(p.cert + 4, 1);
+                }
+            }
+        }
     }
     __syncthreads();   // the shared arrays may be reused for another query
 }
@@ -318,6 +402,7 @@ __device__ __forceinline__ void finalize_query_warp(const FinalizeParams &p, int
         }
     }
     float my_d = kInf;       // lane r: score, later distance, of the r-th candidate
+    float my_s = kInf;       // lane r: its score as the merge left it (for the certificate)
     int32_t my_i = 0x7FFFFFFF;
     int cand_n = 0;
     for (int r = 0; r < want; ++r) {
@@ -356,6 +441,8 @@ __device__ __forceinline__ void finalize_query_warp(const FinalizeParams &p, int
         my_lab = p.labels[my_i];
         my_w = p.weights[my_i];
     }
+    my_s = my_d;
+    float qq = 0.f;          // ||q||^2, every lane
     // ---- exact distances of the candidates, four rows at a time so that their loads overlap; per row the same
     // two partial sums and the same reduction as in finalize_query_cta
     if (p.refine) {
@@ -369,10 +456,15 @@ __device__ __forceinline__ void finalize_query_warp(const FinalizeParams &p, int
                 const int32_t cu = __shfl_sync(0xFFFFFFFFu, my_i, min(j0 + u, cand_n - 1));
                 x[u] = reinterpret_cast<const uint4 *>(reinterpret_cast<const T *>(p.X) + (int64_t)cu * p.dim);
             }
-            float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f};
+            float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f}, n0 = 0.f, n1 = 0.f;
+            const bool with_norm = j0 == 0;
             int c = lane;
             for (; c + 32 < chunks; c += 64) {
                 const uint4 q0 = ld16(q + c), q1 = ld16(q + c + 32);
+                if (with_norm) {
+                    n0 = sqnorm16<T>(q0, n0);
+                    n1 = sqnorm16<T>(q1, n1);
+                }
                 uint4 x0[4], x1[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -387,11 +479,18 @@ __device__ __forceinline__ void finalize_query_warp(const FinalizeParams &p, int
             }
             for (; c < chunks; c += 32) {
                 const uint4 q0 = ld16(q + c);
+                if (with_norm) n0 = sqnorm16<T>(q0, n0);
                 uint4 x0[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) x0[u] = ld16(x[u] + c);
 #pragma unroll
                 for (int u = 0; u < 4; ++u) a0[u] = sqdiff16<T>(q0, x0[u], a0[u]);
+            }
+            if (with_norm) {
+                float nq = n0 + n1;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) nq += __shfl_xor_sync(0xFFFFFFFFu, nq, o);
+                qq = nq;
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -462,14 +561,43 @@ __device__ __forceinline__ void finalize_query_warp(const FinalizeParams &p, int
         }
     }
     const bool hit = k_eff > 0 && (p.rule == FI_HIT_CONF_GT ? best_c > p.tau : best_dwin <= p.tau);
+    const int o = p.out_slot ? p.out_slot[b] : b;
     if (lane == 0) {
-        p.out_label[b] = best_label;
-        p.out_conf[b] = best_c;
-        p.out_hit[b] = hit ? 1 : 0;
+        p.out_label[o] = best_label;
+        p.out_conf[o] = best_c;
+        p.out_hit[o] = hit ? 1 : 0;
     }
     for (int j = lane; j < p.k; j += 32) {
-        if (p.out_topk_dist) p.out_topk_dist[(int64_t)b * p.k + j] = j < k_eff ? d : kInf;
-        if (p.out_topk_idx) p.out_topk_idx[(int64_t)b * p.k + j] = j < k_eff ? ci : -1;
+        if (p.out_topk_dist) p.out_topk_dist[(int64_t)o * p.k + j] = j < k_eff ? d : kInf;
+        if (p.out_topk_idx) p.out_topk_idx[(int64_t)o * p.k + j] = j < k_eff ? ci : -1;
+    }
+    if (p.cert && p.slot_cert) {
+        // same certificate as in finalize_query_cta; lane r still holds the r-th merged score and its exact distance
+        bool ok = true;
+        if (p.refine && k_eff > 0) {
+            const float c_max = __int_as_float(p.cert[3]);
+            const float s_last = __shfl_sync(0xFFFFFFFFu, my_s, cand_n - 1);
+            const float d_k = __shfl_sync(0xFFFFFFFFu, d, k_eff - 1);
+            ok = certified(d_k, s_last, qq, c_max, p.eps, cand_n >= want);
+            float err = lane < cand_n ? fabsf(my_s + qq - my_d) : 0.f;
+#pragma unroll
+            for (int sh = 16; sh > 0; sh >>= 1) err = fmaxf(err, __shfl_xor_sync(0xFFFFFFFFu, err, sh));
+            const float denom = qq + c_max;
+            if (lane == 0 && denom > 0.f && err > 0.f) atomicMax(p.cert + 1, __float_as_int(err / denom));
+        }
+        if (lane == 0) {
+            p.slot_cert[o] = ok ? 1 : 0;
+            if (!ok) {
+                atomicAdd(p.cert, 1);
+                if (p.repair_list) {
+                    const int pos = atomicAdd(p.cert + 2, 1);
+                    if (pos < p.repair_cap) p.repair_list[pos] = b;
+                    else atomicAdd(p.cert + 4, 1);
+                } else {
+                    atomicAdd(p.cert + 4, 1);
+                }
+            }
+        }
     }
 }
 
@@ -727,6 +855,17 @@ fi_status_t launch_finalize(const fi_cache *c, const FinalizeArgs &a, cudaStream
     p.out_hit = a.out.hit;
     p.out_topk_dist = a.out.topk_dist;
     p.out_topk_idx = a.out.topk_idx;
+    // score error model of the distance GEMM: each of its dim / 16 accumulation steps adds to an fp32 partial sum whose
+    // magnitude is at most (||q||^2 + ||c||^2) / 2 and may drop up to one unit in its last place (relative 2^-23; the
+    // accumulation truncates, the errors do not cancel), twice that for the factor -2 in the score; four more steps'
+    // worth covers the rounding of ||c||^2 and of the final subtraction.  Measured on the five workloads the largest
+    // error is about half of this bound at 8,192 to 65,536 values per row.
+    p.eps = ((float)c->cfg.dim / 16.f + 4.f) * 1.1920929e-7f;   // (dim / 16 + 4) * 2^-23
+    p.cert = c->cert_dev;
+    p.slot_cert = c->slot_cert;
+    p.repair_list = a.fill_repair_list ? c->repair_list : nullptr;
+    p.repair_cap = kRepairCap;
+    p.out_slot = a.out_slot;
     // short rows (up to 8 KiB) in batches large enough for the warp-per-query mode; everything else: a CTA per query
     // (the plain kernel needs fewer registers, so more of its CTAs are resident)
     const bool short_rows = (size_t)c->cfg.dim * c->elem_size <= 8192 && a.batch_max >= kWarpModeMinBatch;

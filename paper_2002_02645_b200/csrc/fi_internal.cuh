@@ -14,6 +14,9 @@ constexpr long long kMaxEntries = 2147483647ll - 255;   // cache entries are ind
 constexpr int kStreamMaxBatch = 1; // batches up to this size take the streaming kernel under FI_PATH_AUTO (bf16)
 constexpr int kTileM = 128;        // queries per MMA (= TMEM lanes); a CTA tile holds 128 or 256 queries
 constexpr int kMaxHostStages = 64; // stages a host-driven cascade may have
+constexpr int kRepairCap = 64;     // queries per look-up the exact repair pass can take
+constexpr int kCertWords = 5;      // certificate block: uncertified, max score error (float bits), repair-list length,
+                                   // max ||c||^2 (float bits), uncertified and not repaired
 constexpr int kMaxDevices = 64;    // device ordinals the per-device set-up tables cover
 constexpr int kProfSlots = 256;    // look-ups whose distance-kernel time is kept
 
@@ -190,6 +193,10 @@ struct fi_cache {
                              // CTAs of a GEMM launch (order-preserving integer image of the float)
     fi::GemmPlan *plan_dev;  // written by the GEMM kernel, read by the finalize kernel
     int32_t *status_dev;     // device status word (bounded waits that ran out)
+    int32_t *cert_dev;       // [kCertWords] certificate block of the tensor-core path (see FinalizeParams::cert)
+    uint8_t *slot_cert;      // [max_batch] 1 = the slot's neighbours are proven exact (last look-up)
+    int32_t *repair_list;    // [kRepairCap] slots the exact repair pass looks up again
+    bool repair_on;
     int32_t *calib_acc;      // [2] threshold calibration: max wrong confidence (bit pattern), wrong count
     float *km_dist;          // [max_batch] k-means assignment scratch: nearest distances of one batch (unused output)
     float *km_partial;       // [size x segments x dim] k-means update: per-segment sums of the points of each cluster
@@ -216,7 +223,9 @@ void count_launch(int n = 1);
 fi_status_t check_launch(const char *what);
 
 // ---- launchers (each enqueues on `stream`, returns a status) ----
-fi_status_t launch_row_norms(const void *rows, int dtype, int64_t n, int dim, float *norms, cudaStream_t stream);
+// squared norms of n stored rows; norm_max_bits (nullable) is raised to the largest of them (float bit pattern)
+fi_status_t launch_row_norms(const void *rows, int dtype, int64_t n, int dim, float *norms, int32_t *norm_max_bits,
+                             cudaStream_t stream);
 
 fi_status_t launch_gather_rows(const void *src, int64_t ld_elems, const int32_t *row_idx, int32_t batch_max,
                                const int32_t *count_dev, void *dst, int dim, size_t elem_size, cudaStream_t stream);
@@ -241,6 +250,8 @@ struct FinalizeArgs {
     int list_len;           // entries per list, or -1: read from plan_dev
     int refine;             // 1: scores are approximate, recompute sum (q-c)^2 for the candidates
     fi_lookup_out_t out;
+    const int32_t *out_slot = nullptr;   // nullable: result b is written to output slot out_slot[b]
+    bool fill_repair_list = false;       // uncertified slots are appended to the cache's repair list
 };
 fi_status_t launch_finalize(const fi_cache *c, const FinalizeArgs &a, cudaStream_t stream);
 

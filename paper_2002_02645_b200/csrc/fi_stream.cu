@@ -83,7 +83,8 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // ---------------------------------------------------------------- K0: squared norms of stored rows
 template <typename T>
-__global__ void row_norms_kernel(const T *__restrict__ rows, int64_t n, int dim, float *__restrict__ norms) {
+__global__ void row_norms_kernel(const T *__restrict__ rows, int64_t n, int dim, float *__restrict__ norms,
+                                 int32_t *__restrict__ norm_max_bits) {
     int64_t row = (int64_t)blockIdx.x * (blockDim.x / 32) + (threadIdx.x / 32);
     if (row >= n) return;
     int lane = threadIdx.x & 31;
@@ -92,7 +93,11 @@ __global__ void row_norms_kernel(const T *__restrict__ rows, int64_t n, int dim,
     float s = 0.f;
     for (int c = lane; c < chunks; c += 32) s += Elem<T>::sqnorm(ld_stream16(p + c));
     s = warp_sum(s);
-    if (lane == 0) norms[row] = s;
+    if (lane == 0) {
+        norms[row] = s;
+        // norms are >= 0, so their bit patterns order like the values
+        if (norm_max_bits && s == s) atomicMax(norm_max_bits, __float_as_int(s));
+    }
 }
 
 // ---------------------------------------------------------------- gather rows of the active requests
@@ -221,14 +226,15 @@ stream_lookup_kernel(const T *__restrict__ X, int64_t n_entries, int dim, const 
 
 }  // namespace
 
-fi_status_t launch_row_norms(const void *rows, int dtype, int64_t n, int dim, float *norms, cudaStream_t stream) {
+fi_status_t launch_row_norms(const void *rows, int dtype, int64_t n, int dim, float *norms, int32_t *norm_max_bits,
+                             cudaStream_t stream) {
     if (n <= 0) return FI_OK;
     const int warps = 8;
     unsigned grid = (unsigned)((n + warps - 1) / warps);
     if (dtype == FI_F32)
-        row_norms_kernel<float><<<grid, warps * 32, 0, stream>>>((const float *)rows, n, dim, norms);
+        row_norms_kernel<float><<<grid, warps * 32, 0, stream>>>((const float *)rows, n, dim, norms, norm_max_bits);
     else
-        row_norms_kernel<uint16_t><<<grid, warps * 32, 0, stream>>>((const uint16_t *)rows, n, dim, norms);
+        row_norms_kernel<uint16_t><<<grid, warps * 32, 0, stream>>>((const uint16_t *)rows, n, dim, norms, norm_max_bits);
     count_launch();
     return check_launch("row_norms_kernel");
 }

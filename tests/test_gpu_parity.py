@@ -469,6 +469,76 @@ def test_caches_created_from_two_threads():
         compare_lookup(*got, ref, storage="bf16", tau=0.0, rule=0, cache_labels=st.cache_labels)
 
 
+# ------------------------------------------------------------------ certificate of the tensor-core path, exact repair
+
+def _near_duplicate_case(n, d, b, seed):
+    """Cache rows and requests that are all small perturbations of one vector of large entries: ||q||^2 is about 1e4
+    times the distances, so the rounding of the tensor-core scores is of the order of the gaps between neighbours."""
+    rng = np.random.default_rng(seed)
+    base = 64.0 + 0.5 * rng.integers(0, 8, size=d)                    # exactly representable in bf16 (step 0.5 here)
+    x = (base[None, :] + 0.5 * rng.integers(-2, 3, size=(n, d))).astype(np.float32)
+    q = (base[None, :] + 0.5 * rng.integers(-2, 3, size=(b, d))).astype(np.float32)
+    labels = rng.integers(0, 4, size=n).astype(np.int32)
+    from paper_2002_02645_b200.datagen import StageData, f32_to_bf16_bits
+    xb, qb = f32_to_bf16_bits(x), f32_to_bf16_bits(q)
+    assert (dg.bf16_bits_to_f32(xb) == x).all() and (dg.bf16_bits_to_f32(qb) == q).all()
+    return StageData(d, "bf16", xb, labels, qb)
+
+
+def test_certificate_marks_undecidable_requests_and_repair_makes_them_exact():
+    st = _near_duplicate_case(n=12000, d=1024, b=160, seed=41)
+    k = 5
+    ref = fo.lookup(st.queries, st.cache_vecs, st.cache_labels, k=k, tau=0.0)
+    cache = make_cache(st, k=k, num_classes=4, tau=0.0, max_batch=160, path=fb.FI_PATH_GEMM)
+    cache.read_certificate()                                         # clears whatever the set-up left
+    got = run_lookup(cache, st.queries)
+    flags = cache.slot_certificates(160).numpy().astype(bool)
+    uncertified, unrepaired, err = cache.read_certificate()
+    eps = (1024 / 16 + 4) * 2.0 ** -23
+    print(f"near-duplicate rows: {uncertified} of 160 requests without a certificate, largest score error {err:.3g} "
+          f"(bound used {eps:.3g})")
+    assert uncertified == int((~flags).sum()) == unrepaired and 0 < uncertified <= 160
+    assert 0 < err <= eps                                            # the error model holds on the candidates seen
+    # certified requests are proven exact: they must equal the oracle (the k-th gap exemption apart)
+    sub = np.nonzero(flags)[0]
+    from oracle.fi_oracle import LookupResult
+    pick = lambda r, i: LookupResult(r.label[i], r.conf[i], r.hit[i], r.nd[i], r.ni[i], r.next_d[i])
+    compare_lookup(*[g[sub] for g in got], pick(ref, sub), storage="bf16", tau=0.0, rule=0, cache_labels=st.cache_labels)
+    # with the repair pass every request is either certified or looked up again with exact distances
+    cache.set_repair(True)
+    fixed = run_lookup(cache, st.queries)
+    flags2 = cache.slot_certificates(160).numpy().astype(bool)
+    unc2, unrep2, _ = cache.read_certificate()
+    assert unc2 == uncertified and unrep2 == max(0, uncertified - 64)
+    assert int((~flags2).sum()) == unrep2
+    sub2 = np.nonzero(flags2)[0]
+    stats = compare_lookup(*[g[sub2] for g in fixed], pick(ref, sub2), storage="bf16", tau=0.0, rule=0,
+                           cache_labels=st.cache_labels)
+    print(stats)
+    again = run_lookup(cache, st.queries)
+    for a, b2 in zip(fixed, again):
+        np.testing.assert_array_equal(a, b2)
+    cache.close()
+
+
+def test_certificate_on_ordinary_data_and_streaming_path():
+    w = dg.single_layer(name="t", n_cache=5000, n_query=300, dim=512, num_classes=6, dtype="bf16", sigma=0.6, k=5, seed=43)
+    st = w.stages[0]
+    for path in (fb.FI_PATH_GEMM, fb.FI_PATH_STREAM):
+        cache = make_cache(st, k=5, num_classes=6, tau=0.0, max_batch=300, path=path)
+        cache.read_certificate()
+        run_lookup(cache, st.queries)
+        unc, unrep, err = cache.read_certificate()
+        flags = cache.slot_certificates(300).numpy()
+        print(f"path {path}: uncertified {unc}, largest score error {err:.3g}")
+        assert unc == int((flags == 0).sum())
+        if path == fb.FI_PATH_STREAM:
+            assert unc == 0 and err == 0.0                          # exact distances throughout: nothing to certify
+        else:
+            assert unc < 150 and 0 < err <= (512 / 16 + 4) * 2.0 ** -23
+        cache.close()
+
+
 # ------------------------------------------------------------------ cache rows split over several caches (shards)
 
 @pytest.mark.parametrize("path", [fb.FI_PATH_GEMM, fb.FI_PATH_STREAM])
