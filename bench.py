@@ -875,6 +875,121 @@ def run_projected(args):
         o.close()
 
 
+def run_overlap(args):
+    """Look-ups pipelined with the forward pass (Sec. 5): stage l's look-up runs on its own stream while the main stream
+    already computes layer l + 1.  The layers are stood in for by the caller's own work (one bf16 matrix product per
+    stage on the main stream); the look-up kernels can be limited to a share of the SMs so that both streams make
+    progress.  Two regimes: the config-2 cascade (batch 1,024: the look-ups are tensor-core work themselves) and the
+    config-5 latency look-up (batch 16: the look-up streams the cache at the HBM rate and leaves the tensor cores
+    idle).  Reports, per SM share, the step time against the serial schedule and the fraction of the look-up time
+    that disappears behind the layers."""
+    import torch
+    from paper_2002_02645_b200 import binding as fb
+    from paper_2002_02645_b200 import build as fbuild
+    fbuild.build_library()
+    dev = torch.device("cuda", 0)
+    main, side = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def timed(fn):
+        with torch.cuda.stream(main):
+            for _ in range(max(args.warmup, 3)):
+                fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(main):
+            e0.record(main)
+            for _ in range(args.steps):
+                fn()
+            e1.record(main)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps
+
+    def study(name, caches, begin, lookup, n_stage, m, shares):
+        layer_a = torch.randn(m, m, device=dev, dtype=torch.bfloat16)
+        layer_b = torch.randn(m, m, device=dev, dtype=torch.bfloat16)
+        layer_out = torch.empty(m, m, device=dev, dtype=torch.bfloat16)
+        done = [torch.cuda.Event() for _ in range(n_stage)]
+
+        def layers_only():
+            for _ in range(n_stage):
+                torch.matmul(layer_a, layer_b, out=layer_out)
+
+        def lookups_only():
+            begin()
+            for l in range(n_stage):
+                lookup(l)
+
+        def serial():
+            begin()
+            for l in range(n_stage):
+                torch.matmul(layer_a, layer_b, out=layer_out)       # layer l produces the activations ...
+                lookup(l)                                           # ... which are looked up before layer l + 1 starts
+
+        def pipelined():
+            with torch.cuda.stream(side):
+                side.wait_stream(main)
+                begin()
+            for l in range(n_stage):
+                torch.matmul(layer_a, layer_b, out=layer_out)
+                done[l].record(main)
+                with torch.cuda.stream(side):
+                    side.wait_event(done[l])                        # layer l's activations exist
+                    lookup(l)                                       # runs while the main stream computes layer l + 1
+            main.wait_stream(side)
+
+        t_layers = timed(layers_only)
+        rows = []
+        for sms in shares:
+            for c in caches:
+                c.set_sm_limit(sms)
+            t_look, t_serial, t_pipe = timed(lookups_only), timed(serial), timed(pipelined)
+            rows.append({"lookup_sms": sms or "all", "lookups_alone_ms": t_look, "serial_ms": t_serial, "pipelined_ms": t_pipe,
+                         "lookup_time_hidden": (t_serial - t_pipe) / t_look})
+        for c in caches:
+            c.set_sm_limit(0)
+            c.poll_status()
+        return {"regime": name, "stages": n_stage, "layer_stand_in": f"one {m}^3 bf16 matrix product per stage on the caller's stream",
+                "layers_alone_ms": t_layers, "schedules": rows}
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    out = []
+    # ---- config 2: the 4-stage cascade at batch 1,024
+    w = build_workload("cfg2", seed=0)
+    b0, n_stage = w.stages[0].queries.shape[0], len(w.stages)
+    caches, acts = [], []
+    for s_i, st in enumerate(w.stages):
+        c = fb.FreezeCache(dim=st.dim, capacity=st.cache_vecs.shape[0], num_classes=w.num_classes, k=w.k, dtype=fb.FI_BF16,
+                           max_batch=max(b0, st.calib.shape[0]))
+        c.insert(to_dev(st.cache_vecs, dev), torch.from_numpy(st.cache_labels).to(dev))
+        calibrate(c, to_dev(st.calib, dev), w.meta["percentiles"][s_i])
+        caches.append(c)
+        acts.append(to_dev(st.queries, dev))
+    state = fb.CascadeState(b0, dev)
+    out.append(study("config 2 cascade, batch 1024 (look-ups bound by the tensor cores)", caches,
+                     lambda: fb.cascade_init(state, n_stage), lambda l: fb.cascade_step(caches[l], acts[l], state, l),
+                     n_stage, 6144, (0, 96, 64)))
+    for c in caches:
+        c.close()
+    del caches, acts, w
+    torch.cuda.empty_cache()
+    # ---- config 5: one cache, batch 16, the same look-up after each of four layers
+    w = build_workload("cfg5", seed=0, batch=16)
+    st = w.stages[0]
+    c5 = fb.FreezeCache(dim=st.dim, capacity=st.cache_vecs.shape[0], num_classes=w.num_classes, k=w.k, dtype=fb.FI_BF16,
+                        rule=fb.FI_HIT_DIST_LE, max_batch=16)
+    c5.insert(to_dev(st.cache_vecs, dev), torch.from_numpy(st.cache_labels).to(dev))
+    c5.set_threshold(float("inf"))
+    q5 = to_dev(st.queries, dev)
+    o5 = fb.LookupOut(16, w.k, dev, with_topk=False)
+    out.append(study("config 5 look-up, batch 16 (bound by HBM)", [c5], lambda: None, lambda l: c5.lookup_batch(q5, out=o5),
+                     4, 5120, (0, 96, 64, 32, 16)))
+    c5.close()
+    clocks = sampler.stop()
+    print(json.dumps({"study": "look-ups pipelined with the forward pass", "data": "synthetic", "steps": args.steps,
+                      "regimes": out, "clocks": clocks}))
+
+
 def run_rowshard(args):
     """The 200,000-entry single-layer workload with the cache ROWS split over the ranks (strong scaling: the same
     8,192 requests and the same entries at every N).  Every rank looks all requests up in its rows, one all-gather
@@ -965,7 +1080,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0", "kmeans", "cfg3-rows", "tau-sweep", "cfg2-proj", "launch-check"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0", "kmeans", "cfg3-rows", "tau-sweep", "cfg2-proj", "launch-check", "overlap"])
     ap.add_argument("--no-targets", action="store_true",
                     help="default workload only: skip the config 3 / 4 / 5 measurements that follow the headline")
     ap.add_argument("--cpu-sample", type=int, default=0,
@@ -984,6 +1099,8 @@ def main():
         run_projected(args)
     elif args.workload == "tau-sweep":
         run_tau_sweep(args)
+    elif args.workload == "overlap":
+        run_overlap(args)
     elif args.workload == "cfg3-rows" and args.impl == "ours":
         run_rowshard(args)
     elif args.impl == "reference":

@@ -46,7 +46,7 @@ typedef enum {
 typedef enum { FI_F32 = 0, FI_BF16 = 1 } fi_dtype_t;
 
 /* Hit rule.  FI_HIT_CONF_GT is the paper's: hit iff confidence > threshold, strict (Pseudocode 1,
- * FreezeInference; Sec. 2.1 "exceeds").  FI_HIT_DIST_LE: hit iff the smallest distance among the
+ * FreezeInference; Sec. 2.1).  FI_HIT_DIST_LE: hit iff the smallest distance among the
  * neighbours that carry the winning label is <= threshold (for k = 1: nearest-neighbour distance). */
 typedef enum { FI_HIT_CONF_GT = 0, FI_HIT_DIST_LE = 1 } fi_hit_rule_t;
 
@@ -109,7 +109,7 @@ fi_status_t fi_cache_destroy(fi_cache_t *cache);
  * Y[item]>; with `weights` an entry is the k-means form of Sec. 4, <cluster centre, majority label,
  * fraction of the majority label>.  vecs: [n x dim] device, row-major, contiguous rows; labels: [n] device
  * int32; weights: [n] device float or NULL (= 1.0).  Also computes each row's squared norm.  Asynchronous
- * on the stream; label values are not range-checked on the host (they are opaque to the look-up).
+ * on the stream (which look-ups see the new entries: fi_cache_lookup_view below); label values are not range-checked on the host (they are opaque to the look-up).
  * Errors: CAPACITY when size + n > capacity (nothing is written), INVALID_ARG, CUDA.
  */
 fi_status_t fi_cache_insert(fi_cache_t *cache, const void *vecs, const int32_t *labels, const float *weights,
@@ -121,8 +121,28 @@ fi_status_t fi_cache_set_threshold(fi_cache_t *cache, float tau);
 /* Choose the kernels later look-ups use (fi_path_t).  UNSUPPORTED for FI_PATH_GEMM on a float32 cache. */
 fi_status_t fi_cache_set_path(fi_cache_t *cache, int32_t path);
 
-/* Number of entries currently stored. */
+/* Number of entries stored, counting every insert that has been enqueued. */
 int64_t fi_cache_size(const fi_cache_t *cache);
+
+/*
+ * Inserting into a cache that is being looked up (Sec. 5, incremental cache update: entries are appended while the
+ * cache serves requests).  An insert may run on one stream while look-ups of the same cache run on another.  A look-up
+ * covers a PREFIX of the entries, fixed when it is enqueued: every insert that has completed by then, and every
+ * insert enqueued earlier on the look-up's own stream, up to the first insert that is neither.  Rows behind that
+ * prefix may be in the middle of being written; the kernels never read them (the row count travels as a kernel
+ * argument; the tensor maps cover the whole capacity and never change).  Up to 16 inserts may be in flight per
+ * cache; one more waits on the host for the oldest.
+ * fi_cache_lookup_view: the number of entries the most recent look-up on this cache covered.
+ * Look-ups of one cache still share its scratch and must be ordered among themselves.
+ */
+int64_t fi_cache_lookup_view(const fi_cache_t *cache);
+
+/*
+ * Limit the look-up kernels of this cache to `sms` persistent CTAs (0 = one per SM of the device, the default), so
+ * that another stream's work, such as the next layer of the network (Sec. 5 pipelines cache look-ups with the
+ * forward pass), finds free SMs while a look-up runs.  Takes effect from the next look-up.
+ */
+fi_status_t fi_cache_set_sm_limit(fi_cache_t *cache, int32_t sms);
 
 /* Forget all entries (size becomes 0; capacity and configuration stay).  Asynchronous work already queued on the
  * cache must have been ordered before later inserts by the caller's stream. */
@@ -173,8 +193,8 @@ fi_status_t fi_cascade_init(const fi_cascade_state_t *state, int32_t num_stages,
 /*
  * One layer of FreezeInference (Pseudocode 1) for a whole batch: look up the activations of the requests
  * still alive in this layer's cache; a hit freezes the request (its label, confidence and stage are
- * recorded); the misses are compacted, order kept, into the batch of the next layer (Sec. 5, "reconstruct
- * the batch after each layer to remove the items that have been frozen").
+ * recorded); the misses are compacted, order kept, into the batch of the next layer (Sec. 5: the batch
+ * is rebuilt after each layer without the items frozen there).
  *   stage_acts  [batch0 x ld_elems] device: row r = activation of request r at this layer
  * Needs state->batch0 <= max_batch of the cache.  Asynchronous; the count stays on the device.
  */
@@ -220,8 +240,8 @@ fi_status_t fi_lookup_noalloc(const void *cache_vecs, const int32_t *labels, con
 /*
  * ComputeThresholds of Pseudocode 1 for one layer (Sec. 3.1 (ii)): look up n validation activations in the
  * layer's cache and set THRESHOLDS[layer] to the largest confidence among the look-ups whose label differs from
- * the label the model itself predicted for that item (0 when no look-up is wrong), "ensuring zero error on the
- * validation data".  The look-ups run in batches of at most max_batch; the maximum is formed on the device.
+ * the label the model itself predicted for that item (0 when no look-up is wrong), so that no validation item is frozen
+ * with a wrong label.  The look-ups run in batches of at most max_batch; the maximum is formed on the device.
  *   val_acts   [n x ld_elems] device, dtype of the cache; model_labels [n] device int32 (Y[item])
  *   tau_out    host float, nullable: receives the threshold; wrong_out host int64, nullable: wrong look-ups
  * The cache's threshold is replaced by the result.  Synchronises the stream before returning.

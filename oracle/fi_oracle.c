@@ -6,11 +6,11 @@
  *
  * Everything is fp64 and follows the plain definition, one query at a time:
  *
- *   distance   D[n] = sum_j (q_j - c_nj)^2          Sec. 3: each neighbour tuple carries "its
- *                                                   distance from the input"; squared L2, with
- *                                                   the square root applied on request (metric 1)
- *   neighbours the k smallest under the order (D, n) Sec. 3, "computes k-nearest neighbors ... a
- *                                                   set of k tuples" (ties: smaller index first)
+ *   distance   D[n] = sum_j (q_j - c_nj)^2          Sec. 3: a neighbour tuple is (label, distance
+ *                                                   to the input); squared L2, with the square
+ *                                                   root applied on request (metric 1)
+ *   neighbours the k smallest under the order (D, n) Sec. 3, the k-nearest-neighbour step of the
+ *                                                   look-up API (ties: smaller index first)
  *   vote       for each label i among them:         Sec. 3, the confidence heuristic
  *                S_i = m_i / k
  *                C_i = S_i * sum_{j: label_j = i} w_j / d_j
@@ -20,8 +20,8 @@
  *   hit        rule 0: conf > tau (strict)          Pseudocode 1, FreezeInference
  *              rule 1: d_win <= tau, d_win the smallest distance among the neighbours that carry
  *                      the winning label (for k = 1 the nearest-neighbour distance)
- *   compaction survivors keep their order           Sec. 5, "reconstruct the batch after each layer
- *                                                   to remove the items that have been frozen"
+ *   compaction survivors keep their order           Sec. 5, rebuilding the batch after a layer
+ *                                                   without the items frozen there
  *
  * Readings where the paper is silent: d = 0 gives 1/d = +inf, so an exact copy hits under rule 0
  * for every finite tau (observation O1 of Sec. 2); with fewer than k entries k_eff = min(k, N)

@@ -28,7 +28,7 @@ EXPORTS = ["fi_cache_create", "fi_cache_destroy", "fi_cache_insert", "fi_cache_s
            "fi_projection_create", "fi_projection_destroy", "fi_projection_set_weights", "fi_projection_apply", "fi_projection_poll_status", "fi_projection_set_profiling",
            "fi_projection_read_profile",
            "fi_cascade_step_projected", "fi_cache_set_repair", "fi_cache_read_certificate",
-           "fi_cache_read_slot_certificates", "fi_launch_count", "fi_last_error", "fi_status_string"]
+           "fi_cache_read_slot_certificates", "fi_cache_lookup_view", "fi_cache_set_sm_limit", "fi_launch_count", "fi_last_error", "fi_status_string"]
 
 
 class fi_cache_config_t(ctypes.Structure):
@@ -99,6 +99,9 @@ def load_library(path: Optional[str] = None):
                                                ctypes.POINTER(i64), vp]
     lib.fi_lookup_noalloc.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, i32, ctypes.c_float, vp, i64, i32,
                                       ctypes.POINTER(fi_lookup_out_t), vp]
+    lib.fi_cache_lookup_view.argtypes = [vp]
+    lib.fi_cache_lookup_view.restype = i64
+    lib.fi_cache_set_sm_limit.argtypes = [vp, i32]
     lib.fi_cache_set_repair.argtypes = [vp, i32]
     lib.fi_cache_read_certificate.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(ctypes.c_float)]
     lib.fi_cache_read_slot_certificates.argtypes = [vp, vp, i32]
@@ -223,6 +226,14 @@ class FreezeCache:
 
     def poll_status(self) -> None:
         _check(self._lib.fi_cache_poll_status(self._h))
+
+    # -- fi_cache_lookup_view / fi_cache_set_sm_limit
+    def lookup_view(self) -> int:
+        """Entries the most recent look-up covered (inserts still in flight on another stream are not among them)."""
+        return int(self._lib.fi_cache_lookup_view(self._h))
+
+    def set_sm_limit(self, sms: int) -> None:
+        _check(self._lib.fi_cache_set_sm_limit(self._h, int(sms)))
 
     # -- fi_cache_set_repair / fi_cache_read_certificate / fi_cache_read_slot_certificates
     def set_repair(self, enable: bool) -> None:

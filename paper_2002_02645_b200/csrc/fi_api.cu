@@ -68,6 +68,8 @@ void free_all(fi_cache *c) {
     cudaFree(c->slot_cert);
     cudaFree(c->repair_list);
     cudaFree(c->h2d_stage);
+    for (int i = 0; i < kMaxPending; ++i)
+        if (c->pend_ev[i]) cudaEventDestroy(c->pend_ev[i]);
     if (c->copy_ev) {
         for (int i = 0; i < kMaxHostStages; ++i) cudaEventDestroy(c->copy_ev[i]);
         delete[] c->copy_ev;
@@ -110,6 +112,7 @@ fi_status_t check_part_scratch(const fi_cache *c, size_t entries) {
 fi_status_t lookup_impl(fi_cache *c, const void *queries, int64_t ld, const int32_t *row_idx, int32_t batch_max,
                         const int32_t *count_dev, const fi_lookup_out_t &out, cudaStream_t stream) {
     if (batch_max == 0) return FI_OK;
+    refresh_view(c, stream);
     const int path = resolve_path(c, batch_max);
     FinalizeArgs fa;
     fa.queries = queries;
@@ -210,6 +213,29 @@ fi_status_t status_from_words(fi_cache *const *caches, int n, const int32_t *wor
 
 }  // namespace
 
+// Entries a look-up enqueued now on `stream` may read.  Inserts retire in order: one counts when its event has completed
+// (its rows, labels, weights and norms are then visible to every later launch) or when it was enqueued on `stream`
+// itself (stream order); the first insert that is neither ends the prefix, whatever follows it.
+void refresh_view(fi_cache *c, cudaStream_t stream) {
+    while (c->pend_n > 0) {
+        PendingInsert &p = c->pending[c->pend_head];
+        if (cudaEventQuery(p.ev) != cudaSuccess) {
+            cudaGetLastError();   // "not ready" is an answer, not a failure
+            break;
+        }
+        c->committed = p.size_after;
+        c->pend_head = (c->pend_head + 1) % kMaxPending;
+        --c->pend_n;
+    }
+    int64_t view = c->committed;
+    for (int i = 0; i < c->pend_n; ++i) {
+        const PendingInsert &p = c->pending[(c->pend_head + i) % kMaxPending];
+        if (p.stream != stream) break;
+        view = p.size_after;
+    }
+    c->size = view;
+}
+
 void set_error(const char *fmt, ...) {
     va_list ap;
     va_start(ap, fmt);
@@ -287,6 +313,7 @@ fi_status_t fi_cache_create(const fi_cache_config_t *cfg, fi_cache_t **out) {
         return cuda_fail(cudaGetLastError(), "fi_cache_create: device properties");
     }
     c->sm_count = prop.multiProcessorCount;
+    c->sm_total = prop.multiProcessorCount;
 
     fi_status_t st = FI_OK;
     auto need = [&](fi_status_t s) {
@@ -319,6 +346,10 @@ fi_status_t fi_cache_create(const fi_cache_config_t *cfg, fi_cache_t **out) {
     if (st == FI_OK) need(dev_alloc(&c->plan_dev, 1, "allocating the plan"));
     if (st == FI_OK && bf16)
         need(dev_alloc(&c->row_bound, ((size_t)cfg->max_batch + 256) * gemm_list_len(cfg->k), "allocating the row bounds"));
+    for (int i = 0; i < kMaxPending && st == FI_OK; ++i) {
+        cudaError_t e = cudaEventCreateWithFlags(&c->pend_ev[i], cudaEventDisableTiming);
+        if (e != cudaSuccess) st = cuda_fail(e, "creating the insert events");
+    }
     if (st == FI_OK) need(dev_alloc(&c->status_dev, 1, "allocating the status word"));
     if (st == FI_OK) need(dev_alloc(&c->cert_dev, (size_t)kCertWords, "allocating the certificate block"));
     if (st == FI_OK) need(dev_alloc(&c->slot_cert, (size_t)cfg->max_batch, "allocating the certificate flags"));
@@ -375,8 +406,8 @@ fi_status_t fi_cache_insert(fi_cache_t *c, const void *vecs, const int32_t *labe
         return FI_ERR_INVALID_ARG;
     }
     if (n == 0) return FI_OK;
-    if (c->size + n > c->cfg.capacity) {
-        set_error("fi_cache_insert: %lld entries do not fit (size %lld, capacity %lld)", (long long)n, (long long)c->size,
+    if (c->enqueued + n > c->cfg.capacity) {
+        set_error("fi_cache_insert: %lld entries do not fit (size %lld, capacity %lld)", (long long)n, (long long)c->enqueued,
                   (long long)c->cfg.capacity);
         return FI_ERR_CAPACITY;
     }
@@ -387,24 +418,39 @@ fi_status_t fi_cache_insert(fi_cache_t *c, const void *vecs, const int32_t *labe
     DeviceGuard guard(c->cfg.device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const size_t row_bytes = (size_t)c->cfg.dim * c->elem_size;
-    unsigned char *dst = static_cast<unsigned char *>(c->rows) + (size_t)c->size * row_bytes;
+    // a full ring of inserts in flight: wait for the oldest (the only place an insert blocks the host)
+    if (c->pend_n == kMaxPending) {
+        cudaError_t e0 = cudaEventSynchronize(c->pending[c->pend_head].ev);
+        if (e0 != cudaSuccess) return cuda_fail(e0, "fi_cache_insert: waiting for an earlier insert");
+        c->committed = c->pending[c->pend_head].size_after;
+        c->pend_head = (c->pend_head + 1) % kMaxPending;
+        --c->pend_n;
+    }
+    const int64_t at = c->enqueued;   // the new entries go behind everything enqueued so far
+    unsigned char *dst = static_cast<unsigned char *>(c->rows) + (size_t)at * row_bytes;
     cudaError_t e = cudaMemcpyAsync(dst, vecs, (size_t)n * row_bytes, cudaMemcpyDeviceToDevice, stream);
     if (e != cudaSuccess) return cuda_fail(e, "fi_cache_insert: copying rows");
-    e = cudaMemcpyAsync(c->labels + c->size, labels, (size_t)n * sizeof(int32_t), cudaMemcpyDeviceToDevice, stream);
+    e = cudaMemcpyAsync(c->labels + at, labels, (size_t)n * sizeof(int32_t), cudaMemcpyDeviceToDevice, stream);
     if (e != cudaSuccess) return cuda_fail(e, "fi_cache_insert: copying labels");
     if (weights) {
-        e = cudaMemcpyAsync(c->weights + c->size, weights, (size_t)n * sizeof(float), cudaMemcpyDeviceToDevice, stream);
+        e = cudaMemcpyAsync(c->weights + at, weights, (size_t)n * sizeof(float), cudaMemcpyDeviceToDevice, stream);
         if (e != cudaSuccess) return cuda_fail(e, "fi_cache_insert: copying weights");
     } else {
         int grid = (int)((n + 255) / 256 < 1024 ? (n + 255) / 256 : 1024);
-        fill_f32_kernel<<<grid, 256, 0, stream>>>(c->weights + c->size, n, 1.0f);
+        fill_f32_kernel<<<grid, 256, 0, stream>>>(c->weights + at, n, 1.0f);
         count_launch();
         fi_status_t st = check_launch("fill_f32_kernel");
         if (st != FI_OK) return st;
     }
-    fi_status_t st = launch_row_norms(dst, c->cfg.dtype, n, c->cfg.dim, c->norms + c->size, c->cert_dev + 3, stream);
+    fi_status_t st = launch_row_norms(dst, c->cfg.dtype, n, c->cfg.dim, c->norms + at, c->cert_dev + 3, stream);
     if (st != FI_OK) return st;
-    c->size += n;
+    // the entries become visible to look-ups on other streams when this event has completed
+    const int slot = (c->pend_head + c->pend_n) % kMaxPending;
+    e = cudaEventRecord(c->pend_ev[slot], stream);
+    if (e != cudaSuccess) return cuda_fail(e, "fi_cache_insert: recording the completion event");
+    c->enqueued = at + n;
+    c->pending[slot] = PendingInsert{stream, c->pend_ev[slot], c->enqueued};
+    ++c->pend_n;
     return FI_OK;
 }
 
@@ -430,7 +476,19 @@ fi_status_t fi_cache_set_path(fi_cache_t *c, int32_t path) {
     return FI_OK;
 }
 
-int64_t fi_cache_size(const fi_cache_t *c) { return c ? c->size : 0; }
+int64_t fi_cache_size(const fi_cache_t *c) { return c ? c->enqueued : 0; }
+
+int64_t fi_cache_lookup_view(const fi_cache_t *c) { return c ? c->size : 0; }
+
+fi_status_t fi_cache_set_sm_limit(fi_cache_t *c, int32_t sms) {
+    if (!c || sms < 0) {
+        set_error("fi_cache_set_sm_limit: null cache or negative count");
+        return FI_ERR_INVALID_ARG;
+    }
+    c->sm_limit = sms;
+    c->sm_count = sms > 0 && sms < c->sm_total ? sms : c->sm_total;
+    return FI_OK;
+}
 
 fi_status_t fi_cache_clear(fi_cache_t *c) {
     if (!c) {
@@ -438,6 +496,10 @@ fi_status_t fi_cache_clear(fi_cache_t *c) {
         return FI_ERR_INVALID_ARG;
     }
     c->size = 0;
+    c->enqueued = 0;
+    c->committed = 0;
+    c->pend_n = 0;
+    c->pend_head = 0;
     DeviceGuard guard(c->cfg.device);
     cudaMemsetAsync(c->cert_dev + 3, 0, sizeof(int32_t), nullptr);   // largest norm of the entries held: none now
     return FI_OK;
@@ -451,6 +513,7 @@ fi_status_t fi_kmeans_step(fi_cache_t *c, const void *points, int64_t ld_elems, 
         set_error("fi_kmeans_step: null or negative argument");
         return FI_ERR_INVALID_ARG;
     }
+    refresh_view(c, static_cast<cudaStream_t>(cuda_stream));
     if (c->cfg.k != 1 || c->size <= 0) {
         set_error("fi_kmeans_step: the centres cache must have k = 1 and hold at least one centre");
         return FI_ERR_INVALID_ARG;
@@ -895,6 +958,7 @@ fi_status_t fi_projection_apply(const fi_projection_t *p, const void *x, int64_t
         set_error("fi_projection_apply: null or negative argument");
         return FI_ERR_INVALID_ARG;
     }
+    refresh_view(p->w, static_cast<cudaStream_t>(cuda_stream));
     if (batch_max > p->max_batch || p->w->size != p->out_dim) {
         set_error("fi_projection_apply: batch %d exceeds max_batch %d, or the weights were never set", batch_max, p->max_batch);
         return FI_ERR_INVALID_ARG;

@@ -17,6 +17,7 @@ constexpr int kMaxHostStages = 64; // stages a host-driven cascade may have
 constexpr int kRepairCap = 64;     // queries per look-up the exact repair pass can take
 constexpr int kCertWords = 5;      // certificate block: uncertified, max score error (float bits), repair-list length,
                                    // max ||c||^2 (float bits), uncertified and not repaired
+constexpr int kMaxPending = 16;    // inserts that may be in flight on a cache at once
 constexpr int kMaxDevices = 64;    // device ordinals the per-device set-up tables cover
 constexpr int kProfSlots = 256;    // look-ups whose distance-kernel time is kept
 
@@ -169,10 +170,25 @@ __host__ __device__ inline GemmPlan make_product_plan(int count, long long n_row
 }  // namespace fi
 
 // The cache object behind the opaque handle.
+// An insert whose copies may still be running: the entries count for look-ups on other streams once `ev` has completed.
+struct PendingInsert {
+    cudaStream_t stream;
+    cudaEvent_t ev;
+    int64_t size_after;
+};
+
 struct fi_cache {
     fi_cache_config_t cfg;
-    int64_t size;            // entries stored
-    int sm_count;
+    int64_t size;            // entries the look-up being enqueued covers (refresh_view): every insert that is complete or
+                             // ordered before it on its stream, up to the first one that is neither
+    int64_t enqueued;        // entries whose insert has been enqueued (what fi_cache_size reports)
+    int64_t committed;       // entries of inserts known to be complete
+    PendingInsert pending[fi::kMaxPending];   // oldest first, as a ring
+    int pend_head, pend_n;
+    cudaEvent_t pend_ev[fi::kMaxPending];     // one event per ring slot, created with the cache
+    int sm_limit;            // CTAs the persistent kernels of a look-up may occupy (0 = all SMs)
+    int sm_count;            // CTAs the persistent kernels launch (sm_total, or the caller's limit)
+    int sm_total;            // SMs of the device
     size_t elem_size;
     // device storage owned by the cache
     void *rows;              // [capacity x dim]
@@ -278,6 +294,8 @@ fi_status_t launch_gemm_project(fi_cache *w, const void *queries_compact, int64_
 size_t product_dump_units(int max_batch, int64_t n_rows, int sm_count);
 fi_status_t launch_wait_selftest(fi_cache *c, long long limit_cycles, cudaStream_t stream);
 fi_status_t ensure_tensor_maps(fi_cache *c);
+// sets c->size to the entries a look-up enqueued now on `stream` may read
+void refresh_view(fi_cache *c, cudaStream_t stream);
 size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, int dim);
 // upper bound of gemm_part_entries over every batch <= max_batch and every cache size <= capacity
 size_t gemm_part_entries_bound(int max_batch, int64_t capacity, int sm_count, int k, int dim);

@@ -469,6 +469,64 @@ def test_caches_created_from_two_threads():
         compare_lookup(*got, ref, storage="bf16", tau=0.0, rule=0, cache_labels=st.cache_labels)
 
 
+# ------------------------------------------------------------------ inserts into a cache that is being looked up
+
+@pytest.mark.parametrize("path", [fb.FI_PATH_GEMM, fb.FI_PATH_STREAM])
+def test_inserts_on_one_stream_while_lookups_run_on_another(path):
+    """Sec. 5, incremental cache update.  Entries are appended on one stream while look-ups run on another; every look-up
+    covers a prefix of the entries (reported by lookup_view) and must equal the oracle's answer on exactly that prefix."""
+    n, chunk, d, b, k = 24000, 3000, 2048, 48, 5
+    w = dg.single_layer(name="t", n_cache=n, n_query=b, dim=d, num_classes=6, dtype="bf16", sigma=0.6, k=k, seed=51)
+    st = w.stages[0]
+    cache = fb.FreezeCache(dim=d, capacity=n, num_classes=6, k=k, dtype=fb.FI_BF16, max_batch=b, path=path)
+    xs, ls, q = to_device(st.cache_vecs), torch.from_numpy(st.cache_labels).cuda(), to_device(st.queries)
+    s_ins, s_look = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    seen = []
+    for lo in range(0, n, chunk):
+        with torch.cuda.stream(s_ins):
+            cache.insert(xs[lo:lo + chunk], ls[lo:lo + chunk])
+        assert cache.size() == lo + chunk                      # enqueued entries count at once
+        with torch.cuda.stream(s_look):
+            out = cache.lookup_batch(q)
+            seen.append((cache.lookup_view(), out))
+    torch.cuda.synchronize()
+    out = cache.lookup_batch(q)                                # everything has landed: the whole cache
+    seen.append((cache.lookup_view(), out))
+    torch.cuda.synchronize()
+    cache.poll_status()
+    views = [v for v, _ in seen]
+    print(f"path {path}: look-ups covered {views} entries while {n // chunk} inserts of {chunk} were enqueued")
+    assert views == sorted(views) and views[-1] == n and all(v % chunk == 0 for v in views)
+    assert all(v <= (i + 1) * chunk for i, v in enumerate(views[:-1]))
+    refs = {}
+    for view, out in seen:
+        got = [t.cpu().numpy() for t in (out.label, out.conf, out.hit, out.topk_dist, out.topk_idx)]
+        if view == 0:
+            assert (got[0] == -1).all() and (got[2] == 0).all() and (got[4] == -1).all()
+            continue
+        if view not in refs:
+            refs[view] = fo.lookup(st.queries, st.cache_vecs[:view], st.cache_labels[:view], k=k, tau=0.0)
+        compare_lookup(*got, refs[view], storage="bf16", tau=0.0, rule=0, cache_labels=st.cache_labels[:view])
+    cache.close()
+
+
+def test_lookup_on_a_limited_number_of_sms_gives_the_same_answers():
+    w = dg.single_layer(name="t", n_cache=9000, n_query=600, dim=1024, num_classes=6, dtype="bf16", sigma=0.6, k=5, seed=52)
+    st = w.stages[0]
+    cache = make_cache(st, k=5, num_classes=6, tau=0.0, max_batch=600)
+    full = run_lookup(cache, st.queries)
+    for sms in (40, 7):
+        cache.set_sm_limit(sms)
+        part = run_lookup(cache, st.queries)
+        for a, c in zip(full, part):
+            np.testing.assert_array_equal(a, c)
+    cache.set_sm_limit(0)
+    ref = fo.lookup(st.queries, st.cache_vecs, st.cache_labels, k=5, tau=0.0)
+    compare_lookup(*full, ref, storage="bf16", tau=0.0, rule=0, cache_labels=st.cache_labels)
+    cache.close()
+
+
 # ------------------------------------------------------------------ certificate of the tensor-core path, exact repair
 
 def _near_duplicate_case(n, d, b, seed):
