@@ -130,7 +130,10 @@ __device__ __forceinline__ bool certified(float d_k, float s_last, float qq, flo
 __device__ __forceinline__ bool pair_less(float s, int i, float t, int j) { return s < t || (s == t && i < j); }
 
 // One query, finished by all threads of a CTA together.
-template <typename T>
+// kLong: rows of at least kLongRowChunks 16-byte chunks take the exact distances by slices of the row (below)
+constexpr int kLongRowChunks = 1024;
+
+template <typename T, bool kLong>
 __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int b, int parts, int list_len) {
     __shared__ float cand_s[kMaxK];
     __shared__ float cand_d[kMaxK];
@@ -161,16 +164,24 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
     __shared__ int32_t cand_n_sh;
     const bool head_merge = p.refine != 0 && parts <= 64;
     if (head_merge) {
+        // all entries of the lists come into shared memory in one round trip (every thread of the CTA fetches a few), so
+        // that the merging warp steps through its lists without waiting on global memory between rounds
+        __shared__ int32_t ent_k[64 * kMaxK];
+        __shared__ int32_t ent_i[64 * kMaxK];
+        for (int e = tid; e < entries; e += kFinThreads) {
+            const int ii = pi[e];
+            const bool live = ii >= 0 && ii < p.n_entries;   // else the list has ended (an index past the cache cannot occur; never follow one)
+            ent_k[e] = live ? score_key(ps[e]) : 0x7FFFFFFF;
+            ent_i[e] = live ? ii : 0x7FFFFFFF;
+        }
+        __syncthreads();
         if (warp == 0) {
             auto head = [&](int list, int h, int32_t &k, int32_t &i) {
                 k = 0x7FFFFFFF;
                 i = 0x7FFFFFFF;
                 if (list < parts && h < list_len) {
-                    const int ii = pi[list * list_len + h];
-                    if (ii >= 0 && ii < p.n_entries) {   // else the list has ended (an index past the cache cannot occur; never follow one)
-                        k = score_key(ps[list * list_len + h]);
-                        i = ii;
-                    }
+                    k = ent_k[list * list_len + h];
+                    i = ent_i[list * list_len + h];
                 }
             };
             int h0 = 0, h1 = 0;
@@ -240,42 +251,97 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
         cand_lab[tid] = p.labels[cand_i[tid]];
         cand_w[tid] = p.weights[cand_i[tid]];
     }
-    // ---- exact distances of the candidates
+    // ---- exact distances of the candidates.  The row length is cut into blocks of 32 chunks of 16 bytes; warp w takes
+    // every kFinWarps-th block and, for its blocks, reads the query ONCE and up to eight candidate rows against it
+    // (nine 16-byte loads in flight per lane).  A warp per candidate, each walking the whole query, read the query
+    // eight times over and was bound by the traffic from L2 to the SMs on long rows (2.2 GB for 1,024 requests of
+    // 65,536 values, of which the candidates are 1.07 GB) and by a chain of dependent DRAM round trips on small batches.
+    // The partial sums are added in a fixed order (lanes by shuffle tree, then warps 0..7), so reruns are bit-identical.
     if (p.refine) {
+        constexpr int kGroup = 8;   // candidates per pass over the query
+        __shared__ float part[kFinWarps][kGroup + 1];
         const int64_t qr = p.row_idx ? (int64_t)p.row_idx[b] : (int64_t)b;
-        const T *q = reinterpret_cast<const T *>(p.Q) + qr * p.ldq;
+        const uint4 *q4 = reinterpret_cast<const uint4 *>(reinterpret_cast<const T *>(p.Q) + qr * p.ldq);
         const int chunks = p.dim / (16 / (int)sizeof(T));
-        for (int j = warp; j < cand_n; j += kFinWarps) {
-            const T *x = reinterpret_cast<const T *>(p.X) + (int64_t)cand_i[j] * p.dim;
-            float a0 = 0.f, a1 = 0.f, n0 = 0.f, n1 = 0.f;
-            const bool with_norm = j == 0;   // ||q||^2 for the certificate rides along with the first candidate
-            int c = lane;
-            for (; c + 32 < chunks; c += 64) {
-                uint4 x0 = ld16(reinterpret_cast<const uint4 *>(x) + c);
-                uint4 x1 = ld16(reinterpret_cast<const uint4 *>(x) + c + 32);
-                uint4 q0 = ld16(reinterpret_cast<const uint4 *>(q) + c);
-                uint4 q1 = ld16(reinterpret_cast<const uint4 *>(q) + c + 32);
-                a0 = sqdiff16<T>(q0, x0, a0);
-                a1 = sqdiff16<T>(q1, x1, a1);
-                if (with_norm) {
-                    n0 = sqnorm16<T>(q0, n0);
-                    n1 = sqnorm16<T>(q1, n1);
+        // short rows (fewer than 1,024 chunks: under 16 KiB): a warp per candidate, each walking the whole row, has less
+        // to reduce and no barrier; the traffic argument above only bites on long rows
+        if (!kLong) {
+            const T *q = reinterpret_cast<const T *>(q4);
+            for (int j = warp; j < cand_n; j += kFinWarps) {
+                const T *x = reinterpret_cast<const T *>(p.X) + (int64_t)cand_i[j] * p.dim;
+                float a0 = 0.f, a1 = 0.f, n0 = 0.f, n1 = 0.f;
+                const bool with_norm = j == 0;   // ||q||^2 for the certificate rides along with the first candidate
+                int c = lane;
+                for (; c + 32 < chunks; c += 64) {
+                    uint4 x0 = ld16(reinterpret_cast<const uint4 *>(x) + c);
+                    uint4 x1 = ld16(reinterpret_cast<const uint4 *>(x) + c + 32);
+                    uint4 q0 = ld16(reinterpret_cast<const uint4 *>(q) + c);
+                    uint4 q1 = ld16(reinterpret_cast<const uint4 *>(q) + c + 32);
+                    a0 = sqdiff16<T>(q0, x0, a0);
+                    a1 = sqdiff16<T>(q1, x1, a1);
+                    if (with_norm) {
+                        n0 = sqnorm16<T>(q0, n0);
+                        n1 = sqnorm16<T>(q1, n1);
+                    }
+                }
+                for (; c < chunks; c += 32) {
+                    const uint4 q0 = ld16(reinterpret_cast<const uint4 *>(q) + c);
+                    a0 = sqdiff16<T>(q0, ld16(reinterpret_cast<const uint4 *>(x) + c), a0);
+                    if (with_norm) n0 = sqnorm16<T>(q0, n0);
+                }
+                float a = a0 + a1, nq = n0 + n1;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
+                    nq += __shfl_xor_sync(0xFFFFFFFFu, nq, o);
+                }
+                if (lane == 0) {
+                    cand_d[j] = a;
+                    if (with_norm) qq_sh = nq;
                 }
             }
-            for (; c < chunks; c += 32) {
-                const uint4 q0 = ld16(reinterpret_cast<const uint4 *>(q) + c);
-                a0 = sqdiff16<T>(q0, ld16(reinterpret_cast<const uint4 *>(x) + c), a0);
-                if (with_norm) n0 = sqnorm16<T>(q0, n0);
-            }
-            float a = a0 + a1, nq = n0 + n1;
+        } else {
+            for (int j0 = 0; j0 < cand_n; j0 += kGroup) {
+                const int nj = min(kGroup, cand_n - j0);
+                const uint4 *x[kGroup];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
-                nq += __shfl_xor_sync(0xFFFFFFFFu, nq, o);
-            }
-            if (lane == 0) {
-                cand_d[j] = a;
-                if (with_norm) qq_sh = nq;
+                for (int u = 0; u < kGroup; ++u)
+                    x[u] = reinterpret_cast<const uint4 *>(reinterpret_cast<const T *>(p.X) + (int64_t)cand_i[j0 + min(u, nj - 1)] * p.dim);
+                float a[kGroup], nq = 0.f;
+#pragma unroll
+                for (int u = 0; u < kGroup; ++u) a[u] = 0.f;
+                const bool with_norm = j0 == 0;   // ||q||^2 for the certificate rides along with the first pass
+                for (int c = warp * 32 + lane; c < chunks; c += kFinWarps * 32) {
+                    const uint4 qv = ld16(q4 + c);
+                    uint4 xv[kGroup];
+#pragma unroll
+                    for (int u = 0; u < kGroup; ++u)
+                        if (u < nj) xv[u] = ld16(x[u] + c);
+#pragma unroll
+                    for (int u = 0; u < kGroup; ++u)
+                        if (u < nj) a[u] = sqdiff16<T>(qv, xv[u], a[u]);
+                    if (with_norm) nq = sqnorm16<T>(qv, nq);
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                    for (int u = 0; u < kGroup; ++u) a[u] += __shfl_xor_sync(0xFFFFFFFFu, a[u], o);
+                    nq += __shfl_xor_sync(0xFFFFFFFFu, nq, o);
+                }
+                if (lane == 0) {
+#pragma unroll
+                    for (int u = 0; u < kGroup; ++u) part[warp][u] = a[u];
+                    part[warp][kGroup] = nq;
+                }
+                __syncthreads();
+                if (tid < nj || (tid == kGroup && with_norm)) {
+                    float sum = 0.f;
+#pragma unroll
+                    for (int w = 0; w < kFinWarps; ++w) sum += part[w][tid];
+                    if (tid < nj) cand_d[j0 + tid] = sum;
+                    else qq_sh = sum;
+                }
+                __syncthreads();
             }
         }
     } else {
@@ -369,8 +435,8 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
 }
 
 // One query, finished by one warp: for short rows and few candidate entries (at most 32 x kWarpEntries), where a CTA per
-// query spends its time on barriers and on launching CTAs.  Same steps and the same arithmetic, in the same order,
-// as finalize_query_cta: merge by repeated minimum (entries held in registers, lane l the entries l, l + 32, ...),
+// query spends its time on barriers and on launching CTAs.  Same steps as finalize_query_cta (the exact distances are
+// summed in another order, each within fp32 rounding of the other): merge by repeated minimum (entries held in registers, lane l the entries l, l + 32, ...),
 // exact distances (the warp walks one candidate row after the other), order by (distance, index), vote, hit rule.
 constexpr int kWarpEntries = 16;
 
@@ -443,8 +509,8 @@ __device__ __forceinline__ void finalize_query_warp(const FinalizeParams &p, int
     }
     my_s = my_d;
     float qq = 0.f;          // ||q||^2, every lane
-    // ---- exact distances of the candidates, four rows at a time so that their loads overlap; per row the same
-    // two partial sums and the same reduction as in finalize_query_cta
+    // ---- exact distances of the candidates, four rows at a time so that their loads overlap; two partial sums per row
+    // and lane, then a shuffle tree
     if (p.refine) {
         const int64_t qr = p.row_idx ? (int64_t)p.row_idx[b] : (int64_t)b;
         const uint4 *q = reinterpret_cast<const uint4 *>(reinterpret_cast<const T *>(p.Q) + qr * p.ldq);
@@ -609,7 +675,19 @@ __global__ void __launch_bounds__(kFinThreads) finalize_kernel(FinalizeParams p)
     if (b >= count) return;
     const int parts = p.plan ? p.plan->lists : p.parts;
     const int list_len = p.plan ? p.plan->list_len : p.list_len;
-    finalize_query_cta<T>(p, b, parts, list_len);
+    finalize_query_cta<T, false>(p, b, parts, list_len);
+}
+
+// The same for long rows (16 KiB and more): the slice-wise exact distances hold eight candidates' partial sums per
+// lane, so the kernel is compiled for four CTAs per SM instead of spilling at eight.
+template <typename T>
+__global__ void __launch_bounds__(kFinThreads, 4) finalize_long_kernel(FinalizeParams p) {
+    const int count = p.count_dev ? min(*p.count_dev, p.batch_max) : p.batch_max;
+    const int b = blockIdx.x;
+    if (b >= count) return;
+    const int parts = p.plan ? p.plan->lists : p.parts;
+    const int list_len = p.plan ? p.plan->list_len : p.list_len;
+    finalize_query_cta<T, true>(p, b, parts, list_len);
 }
 
 // Short rows.  Large batches (k-means assignment, threshold calibration) whose candidate entries fit a warp's
@@ -632,7 +710,7 @@ __global__ void __launch_bounds__(kFinThreads) finalize_rows_kernel(FinalizePara
         const int b = blockIdx.x * kFinWarps + warp;
         if (b < count) finalize_query_warp<T>(p, b, parts, list_len, sort_d[warp], sort_i[warp], sort_lab[warp], sort_w[warp]);
     } else if ((int)blockIdx.x < count) {
-        finalize_query_cta<T>(p, blockIdx.x, parts, list_len);
+        finalize_query_cta<T, false>(p, blockIdx.x, parts, list_len);
     }
 }
 
@@ -870,11 +948,14 @@ fi_status_t launch_finalize(const fi_cache *c, const FinalizeArgs &a, cudaStream
     // (the plain kernel needs fewer registers, so more of its CTAs are resident)
     const bool short_rows = (size_t)c->cfg.dim * c->elem_size <= 8192 && a.batch_max >= kWarpModeMinBatch;
     const int grid = a.batch_max;
+    const bool long_rows = a.refine && (size_t)c->cfg.dim * c->elem_size >= (size_t)kLongRowChunks * 16;
     if (c->cfg.dtype == FI_F32) {
         if (short_rows) finalize_rows_kernel<float><<<grid, kFinThreads, 0, stream>>>(p);
+        else if (long_rows) finalize_long_kernel<float><<<grid, kFinThreads, 0, stream>>>(p);
         else finalize_kernel<float><<<grid, kFinThreads, 0, stream>>>(p);
     } else {
         if (short_rows) finalize_rows_kernel<uint16_t><<<grid, kFinThreads, 0, stream>>>(p);
+        else if (long_rows) finalize_long_kernel<uint16_t><<<grid, kFinThreads, 0, stream>>>(p);
         else finalize_kernel<uint16_t><<<grid, kFinThreads, 0, stream>>>(p);
     }
     count_launch();

@@ -250,9 +250,12 @@ def config2(seed: int = 0, shrink: int = 1, n_calib: int = 512, query_seed: Opti
     return w
 
 
-def config3(seed: int = 0, shrink: int = 1, n_calib: int = 512, query_seed: Optional[int] = None) -> Workload:
-    """One layer, 200,000 bf16 entries of 8192 values, sigma 0.7, ReLU; batch 8,192; k = 10."""
-    w = single_layer(name="cfg3_large_cache" + ("" if shrink == 1 else f"_shrink{shrink}"), n_cache=200000 // shrink,
+def config3(seed: int = 0, shrink: int = 1, n_calib: int = 512, query_seed: Optional[int] = None,
+            n_cache: Optional[int] = None) -> Workload:
+    """One layer, 200,000 bf16 entries of 8192 values, sigma 0.7, ReLU; batch 8,192; k = 10.  `n_cache` keeps the batch
+    and takes only the first entries' worth of the cache (profiler captures on a smaller footprint)."""
+    w = single_layer(name="cfg3_large_cache" + ("" if shrink == 1 else f"_shrink{shrink}"),
+                     n_cache=(200000 // shrink) if n_cache is None else n_cache,
                      n_query=8192 // shrink, dim=8192, num_classes=10, dtype="bf16", sigma=0.7, k=10, seed=seed,
                      n_calib=max(1, n_calib // shrink), query_seed=query_seed)
     w.meta.update(rule="conf_gt", percentiles=[50.0])
