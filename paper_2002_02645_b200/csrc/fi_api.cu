@@ -345,7 +345,7 @@ fi_status_t fi_cache_create(const fi_cache_config_t *cfg, fi_cache_t **out) {
     if (st == FI_OK) need(dev_alloc(&c->slot_hit, (size_t)cfg->max_batch, "allocating slot hit flags"));
     if (st == FI_OK) need(dev_alloc(&c->plan_dev, 1, "allocating the plan"));
     if (st == FI_OK && bf16)
-        need(dev_alloc(&c->row_bound, ((size_t)cfg->max_batch + 256) * gemm_list_len(cfg->k), "allocating the row bounds"));
+        need(dev_alloc(&c->row_bound, ((size_t)cfg->max_batch + 512) * gemm_list_len(cfg->k), "allocating the row bounds"));
     for (int i = 0; i < kMaxPending && st == FI_OK; ++i) {
         cudaError_t e = cudaEventCreateWithFlags(&c->pend_ev[i], cudaEventDisableTiming);
         if (e != cudaSuccess) st = cuda_fail(e, "creating the insert events");

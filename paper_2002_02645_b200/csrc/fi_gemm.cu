@@ -25,6 +25,8 @@
 // Every wait is bounded: a wait that runs out sets the cache's status word and the CTA drains and returns.
 #include <cuda_bf16.h>
 
+#include <cstdlib>
+#include <cstring>
 #include <mutex>
 
 #include "fi_internal.cuh"
@@ -115,6 +117,50 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, SmemCt
     }
 }
 
+// ---- pairs of CTAs (cluster of two) working on one tile with tcgen05 in cta_group::2
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
+    uint32_t out;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(addr), "r"(rank));
+    return out;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.aligned;\nbarrier.cluster.wait.aligned;" ::: "memory");
+}
+// arrive on a barrier that may live in the other CTA of the pair (cluster address)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load of a pair: lands in this CTA's shared memory, completes bytes on a barrier of the leader CTA
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar_cluster_addr, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(x), "r"(y)
+        : "memory");
+}
+// one MMA of the pair: D (256 x N, 128 rows in each CTA's TMEM) += A (128 rows per CTA) x B (N/2 rows per CTA)
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+// completion of the pair's MMAs so far, signalled on the barrier at this address in BOTH CTAs
+__device__ __forceinline__ void umma_commit_pair(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(smem_u32(bar)),
+                 "h"((uint16_t)3)
+                 : "memory");
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int x, int y) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
@@ -133,8 +179,8 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t addr) {
     return d;
 }
 // bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n
-__device__ __forceinline__ uint32_t umma_instr_desc(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+__device__ __forceinline__ uint32_t umma_instr_desc(int n, int m = kTileM) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
     asm volatile(
@@ -223,11 +269,13 @@ struct Schedule {
     int cta, num_ctas, m_local, q, num_kb;
     long long n16;
     // ranges mode
-    int col_begin, col_end, tiles, tile_w, first_w, my_groups;
+    int col_begin, col_end, tiles, tile_w, first_w, my_groups, gran;
 
+    // gran: tile widths are multiples of it (16; 32 for pairs, whose CTAs each load half a tile in 16-row boxes)
     __device__ __forceinline__ void setup(const GemmPlan &p, int cta_, int num_ctas_, long long n_entries, int num_kb_,
-                                          bool short_first_tile) {
+                                          bool short_first_tile, int gran_ = 16) {
         plan = p;
+        gran = gran_;
         cta = cta_;
         num_ctas = num_ctas_;
         num_kb = num_kb_;
@@ -250,7 +298,7 @@ struct Schedule {
             // pipeline's serial part.
             first_w = short_first_tile && cols > 3 * kMaxTileN ? kFirstTileN : 0;
             const int rest_tiles = (cols - first_w + kMaxTileN - 1) / kMaxTileN;
-            tile_w = rest_tiles > 0 ? (((cols - first_w + rest_tiles - 1) / rest_tiles + 15) / 16) * 16 : 0;
+            tile_w = rest_tiles > 0 ? (((cols - first_w + rest_tiles - 1) / rest_tiles + gran - 1) / gran) * gran : 0;
             tiles = rest_tiles + (first_w ? 1 : 0);
             my_groups = m_local < p.m_tiles ? (p.m_tiles - m_local + p.mg - 1) / p.mg : 0;
         }
@@ -263,7 +311,9 @@ struct Schedule {
     }
     __device__ __forceinline__ int tile_width(int t) const {
         if (first_w && t == 0) return first_w;
-        const int rest = col_end - tile_col0(t);
+        // (a pair's last tile of the last range may reach up to 16 rows past the end of the cache: those columns score
+        // +inf like every column past the entry count)
+        const int rest = ((col_end - tile_col0(t) + gran - 1) / gran) * gran;
         return rest < tile_w ? rest : tile_w;
     }
     __device__ __forceinline__ int num_items() const {
@@ -324,16 +374,23 @@ struct Schedule {
     }
 };
 
-// MSUB = 128-row MMAs per CTA tile (1 or 2)
-template <int KP, int MSUB>
+// MSUB = 128-row MMAs per CTA tile (1 or 2).  PAIR (with MSUB = 1): the grid is launched as clusters of two CTAs that
+// share every tile: 256 query rows (128 per CTA) against up to 256 cache rows, of which each CTA loads half; the MMAs
+// are issued by the even CTA for both (tcgen05 cta_group::2) and leave each CTA its 128 rows of the accumulator, so the
+// two accumulator buffers of a 128-row tile stay (the select overlaps the next tile's MMAs) while the operand bytes
+// per flop are those of a 256 x 256 tile.  No load is multicast: each CTA fetches its own halves.
+template <int KP, int MSUB, bool PAIR = false>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_x64,
                    const __grid_constant__ CUtensorMap tmap_x16, const float *__restrict__ norms, long long n_entries,
                    int dim, int batch_max, const int32_t *__restrict__ count_dev, int k,
                    float *__restrict__ part_score, int32_t *__restrict__ part_idx, GemmPlan *__restrict__ plan_out,
                    int32_t *row_bound, float *__restrict__ tail_dump, int32_t *__restrict__ status, int product_only) {
-    constexpr int kTileRows = kTileM * MSUB;
+    constexpr int kTileRows = kTileM * MSUB * (PAIR ? 2 : 1);   // query rows per tile (of the CTA, or of the pair)
     constexpr int kATileBytes = kABytes * MSUB;
+    const uint32_t rank = PAIR ? cluster_rank() : 0u;            // 0 = the CTA that issues the pair's MMAs
+    const int worker = PAIR ? (int)blockIdx.x >> 1 : (int)blockIdx.x;
+    const int num_workers = PAIR ? (int)gridDim.x >> 1 : (int)gridDim.x;
     constexpr int kAccBufs = MSUB == 1 ? 2 : 1;   // accumulator sets in TMEM
     constexpr int kSlots = KP;                    // bound slots per query row
 
@@ -351,19 +408,19 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     if (threadIdx.x == 0) {
         int count = count_dev ? min(*count_dev, batch_max) : batch_max;
         if (count < 0) count = 0;
-        ctl->plan = product_only ? make_product_plan(count, n_entries, (int)gridDim.x, kTileRows, num_kb)
-                                 : make_gemm_plan(count, n_entries, (int)gridDim.x, k, kTileRows, num_kb);
+        ctl->plan = product_only ? make_product_plan(count, n_entries, num_workers, kTileRows, num_kb)
+                                 : make_gemm_plan(count, n_entries, num_workers, k, kTileRows, num_kb, PAIR, MSUB == 1 ? 2 : 1);
         ctl->abort_flag = 0;
         if (blockIdx.x == 0) *plan_out = ctl->plan;
     }
     __syncthreads();
     Schedule sched;
-    sched.setup(ctl->plan, (int)blockIdx.x, (int)gridDim.x, n_entries, num_kb, MSUB == 1 && num_kb <= 8);
+    sched.setup(ctl->plan, worker, num_workers, n_entries, num_kb, MSUB == 1 && num_kb <= 8, PAIR ? 32 : 16);
     const GemmPlan &plan = sched.plan;
     const int n_items = sched.num_items();
     if (n_items == 0) return;   // whole CTA, before any barrier
     // as many stages as fit: narrower tiles leave room for a deeper ring
-    const int stage_bytes = kATileBytes + sched.max_width() * (kBlockK * 2);
+    const int stage_bytes = kATileBytes + (PAIR ? sched.max_width() >> 1 : sched.max_width()) * (kBlockK * 2);
     const int num_stages = min(kMaxStages, kStageRegionBytes / stage_bytes);
 
     if (threadIdx.x == 0) {
@@ -373,19 +430,28 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&ctl->tmem_full[a], 1);
-            mbar_init(&ctl->tmem_empty[a], kEpiThreads);
+            mbar_init(&ctl->tmem_empty[a], PAIR ? 2 * kEpiThreads : kEpiThreads);   // a pair: both CTAs' epilogue threads
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
-                     "r"(kTmemCols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            // the same warp of both CTAs, the same destination: the pair gets the same columns in both TMEMs
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                         "r"(kTmemCols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                         "r"(kTmemCols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();   // the other CTA's barriers are initialised before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
@@ -404,18 +470,34 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         ok = false;
                         break;
                     }
-                    mbar_expect_tx(&ctl->full[stage], (uint32_t)(kATileBytes + w * kBlockK * 2));
                     const uint32_t a_dst = smem_u32(stage_base + stage * stage_bytes);
                     const uint32_t b_dst = a_dst + kATileBytes;
+                    if (PAIR) {
+                        // this CTA's 128 query rows and its half of the tile's cache rows; the bytes of both CTAs are
+                        // counted on the leader's barrier, which the leader alone arms
+                        const int hw = w >> 1;
+                        if (rank == 0) mbar_expect_tx(&ctl->full[stage], (uint32_t)(2 * kATileBytes + w * kBlockK * 2));
+                        const uint32_t bar = map_to_rank(smem_u32(&ctl->full[stage]), 0);
 #pragma unroll
-                    for (int ms = 0; ms < MSUB; ++ms)
-                        tma_load_2d(a_dst + ms * kABytes, &tmap_q, &ctl->full[stage], kb * kBlockK,
-                                    m_tile * kTileRows + ms * kTileM);
-                    int r = 0;
-                    for (; r + 64 <= w; r += 64)
-                        tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x64, &ctl->full[stage], kb * kBlockK, col0 + r);
-                    for (; r < w; r += 16)
-                        tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x16, &ctl->full[stage], kb * kBlockK, col0 + r);
+                        for (int ms = 0; ms < MSUB; ++ms)
+                            tma_load_2d_pair(a_dst + ms * kABytes, &tmap_q, bar, kb * kBlockK,
+                                             m_tile * kTileRows + ((int)rank * MSUB + ms) * kTileM);
+                        const int c0 = col0 + (int)rank * hw;
+                        int r = 0;
+                        for (; r + 64 <= hw; r += 64) tma_load_2d_pair(b_dst + r * (kBlockK * 2), &tmap_x64, bar, kb * kBlockK, c0 + r);
+                        for (; r < hw; r += 16) tma_load_2d_pair(b_dst + r * (kBlockK * 2), &tmap_x16, bar, kb * kBlockK, c0 + r);
+                    } else {
+                        mbar_expect_tx(&ctl->full[stage], (uint32_t)(kATileBytes + w * kBlockK * 2));
+#pragma unroll
+                        for (int ms = 0; ms < MSUB; ++ms)
+                            tma_load_2d(a_dst + ms * kABytes, &tmap_q, &ctl->full[stage], kb * kBlockK,
+                                        m_tile * kTileRows + ms * kTileM);
+                        int r = 0;
+                        for (; r + 64 <= w; r += 64)
+                            tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x64, &ctl->full[stage], kb * kBlockK, col0 + r);
+                        for (; r < w; r += 16)
+                            tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x16, &ctl->full[stage], kb * kBlockK, col0 + r);
+                    }
                     if (++stage == (uint32_t)num_stages) {
                         stage = 0;
                         ph ^= 1;
@@ -451,7 +533,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
             uint32_t stage = 0, ph = 0, tile_no = 0;
             bool ok = true;
             // all MMAs of one tile over the k-blocks [kb0, kb1)
@@ -464,7 +546,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kMaxTileN;
-                const uint32_t idesc = umma_instr_desc(w);
+                const uint32_t idesc = umma_instr_desc(w, PAIR ? 2 * kTileM : kTileM);
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait(&ctl->full[stage], ph, ctl, status, 3)) {
                         ok = false;
@@ -475,18 +557,30 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                     const uint64_t bdesc = umma_smem_desc(a_addr + kATileBytes);
 #pragma unroll
                     for (int kk = 0; kk < kBlockK / 16; ++kk) {
+                        if (PAIR) {
 #pragma unroll
-                        for (int ms = 0; ms < MSUB; ++ms)
-                            umma_bf16(d_tmem + ms * kMaxTileN, umma_smem_desc(a_addr + ms * kABytes) + 2 * kk,
-                                      bdesc + 2 * kk, idesc, ((kb - kb0) | kk) != 0);
+                            for (int ms = 0; ms < MSUB; ++ms)
+                                umma_bf16_pair(d_tmem + ms * kMaxTileN, umma_smem_desc(a_addr + ms * kABytes) + 2 * kk,
+                                               bdesc + 2 * kk, idesc, ((kb - kb0) | kk) != 0);
+                        } else {
+#pragma unroll
+                            for (int ms = 0; ms < MSUB; ++ms)
+                                umma_bf16(d_tmem + ms * kMaxTileN, umma_smem_desc(a_addr + ms * kABytes) + 2 * kk,
+                                          bdesc + 2 * kk, idesc, ((kb - kb0) | kk) != 0);
+                        }
                     }
-                    umma_commit(&ctl->empty[stage]);   // frees the stage once these MMAs have read it
+                    // frees the stage once these MMAs have read it (in both CTAs of a pair)
+                    if (PAIR) umma_commit_pair(&ctl->empty[stage]);
+                    else umma_commit(&ctl->empty[stage]);
                     if (++stage == (uint32_t)num_stages) {
                         stage = 0;
                         ph ^= 1;
                     }
                 }
-                if (ok) umma_commit(&ctl->tmem_full[acc]);
+                if (ok) {
+                    if (PAIR) umma_commit_pair(&ctl->tmem_full[acc]);
+                    else umma_commit(&ctl->tmem_full[acc]);
+                }
             };
             if (plan.mode == 0) {
                 for (int g = 0; g < sched.my_groups && ok; ++g)
@@ -509,7 +603,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         const int half = MSUB == 1 ? (ew >> 2) : 0;       // 128-row tiles: which 16-column chunks (even / odd)
         constexpr int kStep = MSUB == 1 ? 32 : 16;        // distance between this warp's chunks
         const int first = half * 16;
-        const int row_in_tile = msub * kTileM + quarter * 32 + lane;
+        const int row_in_tile = ((PAIR ? (int)rank * MSUB : 0) + msub) * kTileM + quarter * 32 + lane;
         const int te = threadIdx.x - kRoleThreads;        // 0..255, queue slot
         float *my_norm = norm_smem + ew * kMaxTileN;      // 256 floats: one buffer (256-row tiles) or two of 128
         // queue slots and norms are read and written through explicit shared-memory addresses
@@ -744,7 +838,8 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             }
             __syncwarp();
             tc_fence_before();
-            mbar_arrive(&ctl->tmem_empty[acc]);
+            if (PAIR) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->tmem_empty[acc]), 0));   // the leader's barrier
+            else mbar_arrive(&ctl->tmem_empty[acc]);
             if (kSlotsAhead && fetched_ahead) load_slots(nx_m_tile, sharing);   // in flight while the queue is drained
             // after the accumulator is released: the MMAs of the next tile can start meanwhile
             if (__any_sync(0xFFFFFFFFu, cnt > 0)) flush(cnt);
@@ -790,7 +885,8 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                 for (int j = 0; j < 16; ++j) dst[(long long)(c0 + j) * kTileRows] = __uint_as_float(v[j]);
             }
             tc_fence_before();
-            mbar_arrive(&ctl->tmem_empty[acc]);
+            if (PAIR) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->tmem_empty[acc]), 0));   // the leader's barrier
+            else mbar_arrive(&ctl->tmem_empty[acc]);
             __syncwarp();
         };
 
@@ -829,9 +925,11 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();   // neither CTA frees its TMEM or leaves while the other may still use it
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -1046,6 +1144,53 @@ fi_status_t launch_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, con
     return check_launch("tail_select_kernel");
 }
 
+// The pair kernel: clusters of two CTAs, one pair per two SMs.
+template <int KP, int MSUB>
+fi_status_t launch_pair_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, const int32_t *count_dev, cudaStream_t stream) {
+    auto kern = gemm_select_kernel<KP, MSUB, true>;
+    if (cudaMemsetAsync(c->row_bound, 0x7F, ((size_t)batch_max + 512) * KP * sizeof(int32_t), stream) != cudaSuccess) {
+        set_error("cannot reset the row bounds");
+        cudaGetLastError();
+        return FI_ERR_CUDA;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3((unsigned)(c->sm_count & ~1), 1, 1);
+    cfg.blockDim = dim3(kGemmThreads, 1, 1);
+    cfg.dynamicSmemBytes = kGemmSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const float *norms = c->norms;
+    long long n = (long long)c->size;
+    int dim = c->cfg.dim, k = c->cfg.k, zero = 0;
+    float *tail = c->tail_dump;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tq, c->tmap_rows64, c->tmap_rows16, norms, n, dim, (int)batch_max, count_dev, k,
+                                       c->part_score, c->part_idx, c->plan_dev, c->row_bound, tail, c->status_dev, zero);
+    count_launch();
+    if (e != cudaSuccess) {
+        set_error("gemm_select_kernel (pairs): %s", cudaGetErrorString(e));
+        cudaGetLastError();
+        return FI_ERR_CUDA;
+    }
+    return check_launch("gemm_select_kernel (pairs)");
+}
+
+template <int MSUB>
+fi_status_t launch_pair(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, const int32_t *count_dev, cudaStream_t stream) {
+    switch (gemm_list_len(c->cfg.k)) {
+        case 4: return launch_pair_kp<4, MSUB>(c, tq, batch_max, count_dev, stream);
+        case 8: return launch_pair_kp<8, MSUB>(c, tq, batch_max, count_dev, stream);
+        case 16: return launch_pair_kp<16, MSUB>(c, tq, batch_max, count_dev, stream);
+        default: return launch_pair_kp<32, MSUB>(c, tq, batch_max, count_dev, stream);
+    }
+}
+
 template <int MSUB>
 fi_status_t launch_msub(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, const int32_t *count_dev, bool tail_possible,
                         cudaStream_t stream) {
@@ -1105,6 +1250,10 @@ fi_status_t prepare_gemm_kernels(int device) {
     prep(gemm_select_kernel<8, 2>);
     prep(gemm_select_kernel<16, 2>);
     prep(gemm_select_kernel<32, 2>);
+    prep(gemm_select_kernel<4, 1, true>);
+    prep(gemm_select_kernel<8, 1, true>);
+    prep(gemm_select_kernel<16, 1, true>);
+    prep(gemm_select_kernel<32, 1, true>);
     if (st == FI_OK) done[device] = true;
     return st;
 }
@@ -1160,6 +1309,26 @@ static bool tail_mode_possible(const fi_cache *c, int batch_max) {
     return false;
 }
 
+// Pairs of CTAs (tcgen05 cta_group::2).  Measured against single CTAs on one B200: a pair keeps two accumulator buffers
+// under a 256-row tile, so the select overlaps the next tile's MMAs, which pays where a tile's k-loop is short enough for
+// the select to be a large share of it and long enough for the hand-over between the two CTAs not to matter: rows of
+// 1,024 to 2,048 values (100,000 entries, batch 4,096: -4 % and -13 %).  On shorter rows the hand-over costs more than
+// the overlap gains, on longer rows the exposed select is a few per cent and the pair's MMAs run 5-8 % slower (one
+// issuing thread and one full-barrier for two SMs), and shapes in wave + tail mode want one deep tile per CTA.
+// (The kernel also runs with 256 query rows per CTA of a pair, a third fewer operand bytes per flop and one accumulator
+// buffer; forced on, it lost 5 % on 8,192-value rows and more elsewhere, so no launch path instantiates it.)
+// FICACHE_PAIR=0 / 1 in the environment overrides the choice (for A/B measurements).
+static bool use_pair_kernel(const fi_cache *c, int batch_max) {
+    static const int forced = [] {
+        const char *e = getenv("FICACHE_PAIR");
+        return e ? atoi(e) : -1;
+    }();
+    if (batch_max <= kTileM || c->sm_count < 2 || c->size < 512) return false;
+    if (forced >= 0) return forced == 1;
+    const int num_kb = (c->cfg.dim + kBlockK - 1) / kBlockK;
+    return num_kb >= 16 && num_kb <= 32 && batch_max >= 8 * kTileM && c->size >= 32768 && !tail_mode_possible(c, batch_max);
+}
+
 fi_status_t launch_gemm_select(fi_cache *c, const void *queries_compact, int64_t ld_elems, int32_t batch_max,
                                const int32_t *count_dev, cudaStream_t stream) {
     if (batch_max <= 0) return FI_OK;
@@ -1182,6 +1351,7 @@ fi_status_t launch_gemm_select(fi_cache *c, const void *queries_compact, int64_t
         set_error("the distance GEMM's partial-sum buffer is missing (%zu slots, %d needed)", c->tail_dump_units, c->sm_count);
         return FI_ERR_CAPACITY;
     }
+    if (use_pair_kernel(c, batch_max)) return launch_pair<1>(c, tq, batch_max, count_dev, stream);
     if (gemm_tile_m(batch_max, c->cfg.dim) == kTileM) return launch_msub<1>(c, tq, batch_max, count_dev, false, stream);
     return launch_msub<2>(c, tq, batch_max, count_dev, tail_possible, stream);
 }

@@ -55,8 +55,10 @@ struct GemmPlan {
     int32_t pieces;       // pieces: tail_tiles * tail_slices
 };
 
+// `pair`: the workers are pairs of CTAs that share one tile of tile_m rows (half each; pair_lists epilogue warps, hence
+// lists, per row; ranges only, range lengths a multiple of 32 rows); num_ctas is then the number of pairs.
 __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entries, int num_ctas, int k, int tile_m,
-                                                   int num_kb) {
+                                                   int num_kb, bool pair = false, int pair_lists = 2) {
     GemmPlan p;
     p.count = count;
     p.m_tiles = (count + tile_m - 1) / tile_m;
@@ -70,10 +72,10 @@ __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entrie
     if (p.m_tiles <= 0 || n16 <= 0) {
         p.mg = p.groups = p.parts = 1;
         p.range16 = 0;
-        p.lists = tile_m == kTileM ? 2 : 1;
+        p.lists = pair ? pair_lists : tile_m == kTileM ? 2 : 1;
         return p;
     }
-    if (tile_m == 2 * kTileM && num_kb >= 64) {
+    if (tile_m == 2 * kTileM && num_kb >= 64 && !pair) {
         const long long nt = (n16 + 15) / 16;                 // tiles of at most 256 rows
         const long long total = (long long)p.m_tiles * nt;
         if (total > num_ctas && total <= num_ctas + num_ctas / 2) {
@@ -94,7 +96,7 @@ __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entrie
     // Few cache rows (one tile spans them all) under many query tiles, e.g. assigning points to k-means centres:
     // cutting the rows into ranges would leave tiles a few rows wide, which the MMAs run at a fraction of their
     // rate while every CTA re-reads the query tiles.  The query tiles are dealt round-robin to all CTAs instead.
-    if (n16 <= 16 && p.m_tiles >= num_ctas / 2) {
+    if (n16 <= 16 && p.m_tiles >= num_ctas / 2 && !pair) {
         p.mg = p.m_tiles < num_ctas ? p.m_tiles : num_ctas;
         p.groups = (p.m_tiles + p.mg - 1) / p.mg;
         p.parts = 1;
@@ -131,12 +133,13 @@ __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entrie
     p.groups = (p.m_tiles + p.mg - 1) / p.mg;
     int parts = num_ctas / p.mg;
     if (parts > n16i) parts = n16i;
-    const int r16 = (n16i + parts - 1) / parts;
+    int r16 = (n16i + parts - 1) / parts;
+    if (pair) r16 += r16 & 1;         // ranges of whole 32-row blocks: each CTA of a pair loads half of every tile
     parts = (n16i + r16 - 1) / r16;   // drop ranges that would be empty
     p.parts = (int32_t)parts;
     p.range16 = (int32_t)r16;
-    // with 128-row tiles two epilogue warps share each row and keep a list each
-    p.lists = p.parts * (tile_m == kTileM ? 2 : 1);
+    // with 128-row tiles (and with pairs) two epilogue warps share each row and keep a list each
+    p.lists = p.parts * (pair ? pair_lists : tile_m == kTileM ? 2 : 1);
     return p;
 }
 

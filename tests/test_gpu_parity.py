@@ -102,6 +102,8 @@ def test_stream_path_large_dim_reads_queries_in_place():
     (12345, 256, 2000, 5),     # short rows, 16 query tiles x 9 long ranges: short first tile, bounds fetched a tile ahead
     (20011, 512, 1100, 10),    # the same with list length 16 (bound slots read on the spot), ragged N and M
     (9000, 320, 2048, 1),      # the same with list length 4, K = 5 blocks
+    (33000, 1024, 1100, 5),    # rows of 1,024 values, many entries, batch above 1,024: pairs of CTAs share 256-row tiles
+    (40001, 2048, 1024, 10),   # the same with list length 16, ragged entry count, 4 query tiles of a pair exactly
 ])
 def test_gemm_path(n, d, b, k):
     w = dg.single_layer(name="t", n_cache=n, n_query=b, dim=d, num_classes=9, dtype="bf16", sigma=0.6, k=k, seed=5)
