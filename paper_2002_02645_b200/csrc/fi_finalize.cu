@@ -209,17 +209,50 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
         __syncthreads();
         cand_n = cand_n_sh;
     }
+    // up to kKeep entries per thread are fetched once and kept in registers for all rounds (a batch of 16 against 296
+    // lists of 4 re-read them from L2 in every round before); longer inputs are read again in each round
+    constexpr int kKeep = 8;
+    const bool kept = !head_merge && entries <= kKeep * kFinThreads;
+    int32_t ck[kKeep], ci[kKeep];
+    if (kept) {
+#pragma unroll
+        for (int j = 0; j < kKeep; ++j) {
+            const int e = tid + j * kFinThreads;
+            ck[j] = 0x7FFFFFFF;
+            ci[j] = 0x7FFFFFFF;
+            if (e < entries) {
+                const int i = pi[e];
+                if (i >= 0 && i < p.n_entries) {   // else: empty slot (an index past the cache cannot occur; never follow one)
+                    ck[j] = score_key(ps[e]);
+                    ci[j] = i;
+                }
+            }
+        }
+    }
     for (int r = 0; r < want && !head_merge; ++r) {
         int32_t best_k = 0x7FFFFFFF;
         int best_i = 0x7FFFFFFF;
-        for (int e = tid; e < entries; e += kFinThreads) {
-            const int i = pi[e];
-            if (i < 0 || i >= p.n_entries) continue;   // empty slot (an index past the cache cannot occur; never follow one)
-            const int32_t k = score_key(ps[e]);
-            const bool above = r == 0 || k > prev_k || (k == prev_k && i > prev_i);
-            if (above && (k < best_k || (k == best_k && i < best_i))) {
-                best_k = k;
-                best_i = i;
+        if (kept) {
+#pragma unroll
+            for (int j = 0; j < kKeep; ++j) {
+                const int32_t k = ck[j];
+                const int i = ci[j];
+                const bool above = r == 0 || k > prev_k || (k == prev_k && i > prev_i);
+                if (i != 0x7FFFFFFF && above && (k < best_k || (k == best_k && i < best_i))) {
+                    best_k = k;
+                    best_i = i;
+                }
+            }
+        } else {
+            for (int e = tid; e < entries; e += kFinThreads) {
+                const int i = pi[e];
+                if (i < 0 || i >= p.n_entries) continue;   // empty slot (an index past the cache cannot occur; never follow one)
+                const int32_t k = score_key(ps[e]);
+                const bool above = r == 0 || k > prev_k || (k == prev_k && i > prev_i);
+                if (above && (k < best_k || (k == best_k && i < best_i))) {
+                    best_k = k;
+                    best_i = i;
+                }
             }
         }
         int32_t mk = __reduce_min_sync(0xFFFFFFFFu, best_k);
