@@ -201,6 +201,10 @@ def build_workload(name: str, seed: int, query_seed=None, batch=16):
         w = dg.config3(seed=seed, query_seed=query_seed, n_cache=50000)
         w.name = "cfg3_quarter_cache"
         return w
+    if name == "cfg4-s3":          # last stage of cfg4 alone (100,000 x 2,048, batch 4,096): the pair kernel's case
+        w = dg.config4(seed=seed, query_seed=query_seed, stages=1, first_stage=3)
+        w.name = "cfg4_stage3_only"
+        return w
     if name == "cfg2-small":       # same recipe, 1/16 of the sizes: a quick functional run
         return dg.config2(seed=seed, shrink=16, query_seed=query_seed)
     if name == "cfg2-s0":          # first stage of cfg2 alone (10,000 x 65536, batch 1,024): the dominant GEMM
@@ -1084,7 +1088,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg3-quarter", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0", "kmeans", "cfg3-rows", "tau-sweep", "cfg2-proj", "launch-check", "overlap"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg3-quarter", "cfg4", "cfg5", "cfg2-small", "cfg2-s0", "cfg4-s0", "cfg4-s3", "kmeans", "cfg3-rows", "tau-sweep", "cfg2-proj", "launch-check", "overlap"])
     ap.add_argument("--no-targets", action="store_true",
                     help="default workload only: skip the config 3 / 4 / 5 measurements that follow the headline")
     ap.add_argument("--cpu-sample", type=int, default=0,

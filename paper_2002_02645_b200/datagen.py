@@ -263,13 +263,14 @@ def config3(seed: int = 0, shrink: int = 1, n_calib: int = 512, query_seed: Opti
 
 
 def config4(seed: int = 0, shrink: int = 1, n_calib: int = 512, query_seed: Optional[int] = None,
-            stages: int = 4) -> Workload:
-    """Four-stage ImageNet-shaped cascade: 100,000 entries per stage, 1,000 Zipf(1.1) classes, sigma 0.6; k = 5."""
+            stages: int = 4, first_stage: int = 0) -> Workload:
+    """Four-stage ImageNet-shaped cascade: 100,000 entries per stage, 1,000 Zipf(1.1) classes, sigma 0.6; k = 5.
+    `first_stage` / `stages` cut out a run of stages (one stage alone: a profiler capture of its kernel)."""
     w = cascade(name="cfg4_imagenet_cascade" + ("" if shrink == 1 else f"_shrink{shrink}"),
-                dims=[256, 512, 1024, 2048][:stages], scales=[0.6] * stages, kind="relu_mixture", n_cache=100000 // shrink,
+                dims=[256, 512, 1024, 2048][first_stage:first_stage + stages], scales=[0.6] * stages, kind="relu_mixture", n_cache=100000 // shrink,
                 n_query=4096 // shrink, n_calib=max(1, n_calib // shrink), num_classes=1000, dtype="bf16", k=5,
                 seed=seed, zipf=1.1, query_seed=query_seed)
-    w.meta.update(rule="conf_gt", percentiles=[80.0, 60.0, 40.0, 20.0][:stages])
+    w.meta.update(rule="conf_gt", percentiles=[80.0, 60.0, 40.0, 20.0][first_stage:first_stage + stages])
     return w
 
 
