@@ -259,6 +259,7 @@ struct TopList {
 // after the last); the others store their partial sums for the tail kernel.
 struct WorkItem {
     int m_tile, col0, w, kb0, kb1;
+    int rows128;     // 128-row MMAs this item takes (256-row tiles: 1 when only the first 128 rows hold requests)
     int list;        // list index the rows' candidates go to (select tiles)
     int dump_slot;   // slot of the partial sums (tail pieces)
     bool select, reset, emit;
@@ -270,6 +271,8 @@ struct Schedule {
     long long n16;
     // ranges mode
     int col_begin, col_end, tiles, tile_w, first_w, my_groups, gran;
+    // spans mode: this CTA's (cache-row tile, k-block) pairs [span0, span1) of query tile span_m
+    int span0, span1, span_m;
 
     // gran: tile widths are multiples of it (16; 32 for pairs, whose CTAs each load half a tile in 16-row boxes)
     __device__ __forceinline__ void setup(const GemmPlan &p, int cta_, int num_ctas_, long long n_entries, int num_kb_,
@@ -302,6 +305,12 @@ struct Schedule {
             tiles = rest_tiles + (first_w ? 1 : 0);
             my_groups = m_local < p.m_tiles ? (p.m_tiles - m_local + p.mg - 1) / p.mg : 0;
         }
+        span0 = span1 = span_m = 0;
+        int j, cm;
+        if (p.mode == 3 && span_owner(p, cta, span_m, j, cm)) {
+            span0 = span_begin(p, num_kb, j, cm);
+            span1 = span_begin(p, num_kb, j + 1, cm);
+        }
     }
     // widest tile this CTA will load (sizes the shared-memory stages)
     __device__ __forceinline__ int max_width() const { return plan.mode == 0 ? tile_w : kMaxTileN; }
@@ -320,6 +329,7 @@ struct Schedule {
         if (plan.m_tiles == 0 || n16 == 0) return 0;
         if (plan.mode == 0) return my_groups * tiles;
         if (plan.mode == 2) return cta < plan.pieces ? (plan.pieces - cta + num_ctas - 1) / num_ctas : 0;
+        if (plan.mode == 3) return span1 > span0 ? (span1 - 1) / num_kb - span0 / num_kb + 1 : 0;
         return 1 + (cta < plan.tail_tiles * plan.tail_slices ? 1 : 0);
     }
     // wave + tail: the id-th tile in (cache-row tile, query tile) order; cache-row tiles are as even as 16-row
@@ -327,6 +337,7 @@ struct Schedule {
     __device__ __forceinline__ void tile_of(int id, WorkItem &it) const {
         const int n = id / plan.m_tiles;
         it.m_tile = id % plan.m_tiles;
+        it.rows128 = 2;
         const long long b0 = n16 * n / plan.n_tiles, b1 = n16 * (n + 1) / plan.n_tiles;
         it.col0 = (int)(b0 * 16);
         it.w = (int)((b1 - b0) * 16);
@@ -336,6 +347,7 @@ struct Schedule {
     // hand-over path between tiles)
     __device__ __forceinline__ void item(int idx, int g, int t, WorkItem &it) const {
         it.dump_slot = 0;
+        it.rows128 = 2;
         if (plan.mode == 0) {
             it.m_tile = g * plan.mg + m_local;
             it.col0 = tile_col0(t);
@@ -356,6 +368,16 @@ struct Schedule {
             it.kb1 = (int)((long long)num_kb * (sl + 1) / plan.tail_slices);
             it.select = it.reset = it.emit = false;
             it.dump_slot = piece;
+            return;
+        }
+        if (plan.mode == 3) {
+            const int n = span0 / num_kb + idx;
+            tile_of(n * plan.m_tiles + span_m, it);
+            it.rows128 = plan.half && span_m == plan.m_tiles - 1 ? 1 : 2;
+            it.kb0 = idx == 0 ? span0 - n * num_kb : 0;
+            it.kb1 = min(num_kb, span1 - n * num_kb);
+            it.select = it.reset = it.emit = false;
+            it.dump_slot = cta * kMaxSpanItems + idx;
             return;
         }
         if (idx == 0) {
@@ -464,7 +486,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             uint32_t issued = 0, stage = 0, ph = 0;
             bool ok = true;
             // all k-blocks [kb0, kb1) of one tile
-            auto load_tile = [&](int m_tile, int col0, int w, int kb0, int kb1) {
+            auto load_tile = [&](int m_tile, int col0, int w, int kb0, int kb1, int rows128) {
                 for (int kb = kb0; kb < kb1; ++kb, ++issued) {
                     if (!mbar_wait(&ctl->empty[stage], ph ^ 1, ctl, status, 1)) {
                         ok = false;
@@ -487,11 +509,12 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         for (; r + 64 <= hw; r += 64) tma_load_2d_pair(b_dst + r * (kBlockK * 2), &tmap_x64, bar, kb * kBlockK, c0 + r);
                         for (; r < hw; r += 16) tma_load_2d_pair(b_dst + r * (kBlockK * 2), &tmap_x16, bar, kb * kBlockK, c0 + r);
                     } else {
-                        mbar_expect_tx(&ctl->full[stage], (uint32_t)(kATileBytes + w * kBlockK * 2));
+                        mbar_expect_tx(&ctl->full[stage], (uint32_t)((MSUB == 2 ? rows128 * kABytes : kATileBytes) + w * kBlockK * 2));
 #pragma unroll
                         for (int ms = 0; ms < MSUB; ++ms)
-                            tma_load_2d(a_dst + ms * kABytes, &tmap_q, &ctl->full[stage], kb * kBlockK,
-                                        m_tile * kTileRows + ms * kTileM);
+                            if (ms < rows128)
+                                tma_load_2d(a_dst + ms * kABytes, &tmap_q, &ctl->full[stage], kb * kBlockK,
+                                            m_tile * kTileRows + ms * kTileM);
                         int r = 0;
                         for (; r + 64 <= w; r += 64)
                             tma_load_2d(b_dst + r * (kBlockK * 2), &tmap_x64, &ctl->full[stage], kb * kBlockK, col0 + r);
@@ -507,12 +530,12 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             if (plan.mode == 0) {
                 for (int g = 0; g < sched.my_groups && ok; ++g)
                     for (int t = 0; t < sched.tiles && ok; ++t)
-                        load_tile(g * plan.mg + sched.m_local, sched.tile_col0(t), sched.tile_width(t), 0, num_kb);
+                        load_tile(g * plan.mg + sched.m_local, sched.tile_col0(t), sched.tile_width(t), 0, num_kb, MSUB);
             } else {
                 for (int idx = 0; idx < n_items && ok; ++idx) {
                     WorkItem it;
                     sched.item(idx, 0, 0, it);
-                    load_tile(it.m_tile, it.col0, it.w, it.kb0, it.kb1);
+                    load_tile(it.m_tile, it.col0, it.w, it.kb0, it.kb1, it.rows128);
                 }
             }
             if (!ok) {
@@ -537,7 +560,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             uint32_t stage = 0, ph = 0, tile_no = 0;
             bool ok = true;
             // all MMAs of one tile over the k-blocks [kb0, kb1)
-            auto mma_tile = [&](int w, int kb0, int kb1) {
+            auto mma_tile = [&](int w, int kb0, int kb1, int rows128) {
                 const uint32_t acc = tile_no % kAccBufs, acc_ph = (tile_no / kAccBufs) & 1;
                 ++tile_no;
                 if (!mbar_wait(&ctl->tmem_empty[acc], acc_ph ^ 1, ctl, status, 2)) {
@@ -565,8 +588,9 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
                         } else {
 #pragma unroll
                             for (int ms = 0; ms < MSUB; ++ms)
-                                umma_bf16(d_tmem + ms * kMaxTileN, umma_smem_desc(a_addr + ms * kABytes) + 2 * kk,
-                                          bdesc + 2 * kk, idesc, ((kb - kb0) | kk) != 0);
+                                if (ms < rows128)
+                                    umma_bf16(d_tmem + ms * kMaxTileN, umma_smem_desc(a_addr + ms * kABytes) + 2 * kk,
+                                              bdesc + 2 * kk, idesc, ((kb - kb0) | kk) != 0);
                         }
                     }
                     // frees the stage once these MMAs have read it (in both CTAs of a pair)
@@ -585,12 +609,12 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             if (plan.mode == 0) {
                 for (int g = 0; g < sched.my_groups && ok; ++g)
                     for (int t = 0; t < sched.tiles && ok; ++t)
-                        mma_tile(sched.tile_width(t), 0, num_kb);
+                        mma_tile(sched.tile_width(t), 0, num_kb, MSUB);
             } else {
                 for (int idx = 0; idx < n_items && ok; ++idx) {
                     WorkItem it;
                     sched.item(idx, 0, 0, it);
-                    mma_tile(it.w, it.kb0, it.kb1);
+                    mma_tile(it.w, it.kb0, it.kb1, it.rows128);
                 }
             }
         }
@@ -876,7 +900,8 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             if (!ok) return;
             tc_fence_after();
             float *dst = tail_dump + ((long long)it.dump_slot * kMaxTileN) * kTileRows + row_in_tile;
-            for (int c0 = first; c0 < it.w; c0 += kStep) {
+            // (the warps of a 128-row half that took no MMA only keep the barrier counts)
+            for (int c0 = first; c0 < it.w && msub < it.rows128; c0 += kStep) {
                 uint32_t v[16];
                 __syncwarp();
                 tmem_ld16(taddr + c0, v);
@@ -933,70 +958,247 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     }
 }
 
-// Wave + tail mode, step 1: add up the pieces of every tail tile and turn the dot products into scores, in place
-// in the first piece's slot.  Grid (tail tiles, 16 column groups), one query row per thread; the partial sums are
-// column-major, so a warp reads 128 contiguous bytes.  Pieces are added in their order: the sum does not depend on
-// timing.
-__global__ void __launch_bounds__(2 * kTileM)
-tail_reduce_kernel(const GemmPlan *__restrict__ plan_dev, int num_ctas, float *__restrict__ tail_dump,
-                   const float *__restrict__ norms, long long n_entries) {
-    const GemmPlan plan = *plan_dev;
-    if (plan.mode != 1 || (int)blockIdx.x >= plan.tail_tiles) return;
-    constexpr int kRows = 2 * kTileM;
-    const long long n16 = (n_entries + 15) / 16;
-    const int n = (num_ctas + (int)blockIdx.x) / plan.m_tiles;
-    const long long b0 = n16 * n / plan.n_tiles, b1 = n16 * (n + 1) / plan.n_tiles;
-    const int col0 = (int)(b0 * 16), w = (int)((b1 - b0) * 16);
-    const int c0 = blockIdx.y * 16;
-    if (c0 >= w) return;
-    float *base = tail_dump + ((long long)blockIdx.x * plan.tail_slices * kMaxTileN + c0) * kRows + threadIdx.x;
-    float dot[16];
-#pragma unroll
-    for (int j = 0; j < 16; ++j) dot[j] = 0.f;
-    for (int sl = 0; sl < plan.tail_slices; ++sl) {
-        const float *p = base + (long long)sl * kMaxTileN * kRows;
-#pragma unroll
-        for (int j = 0; j < 16; ++j) dot[j] += p[j * kRows];
-    }
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        const int c = col0 + c0 + j;
-        const float nrm = (long long)c < n_entries ? __ldg(norms + c) : __int_as_float(0x7F800000);
-        base[j * kRows] = fmaf(-2.f, dot[j], nrm);
-    }
-}
-
-// Step 2: per-row select over the scores of a tail tile.  One CTA per tail tile, one query row per thread.
+// Wave + tail and spans modes: add up the pieces of a tile in their order (the sum does not depend on timing), turn
+// the dot products into scores and select per row.  A CTA takes 32 query rows of one tile and one warp per share of
+// the tile's columns (a warp reads 128 contiguous bytes of the column-major partial sums per column; with a share of
+// 16 columns per thread the loads of one piece are all in flight at once, and there are enough threads to cover the
+// latency of memory).
+//
+// Lists of up to 8 entries (16 shares of 16 columns): no thread sorts anything.  The smallest scores of the 16 shares
+// of a row are 16 different columns, so the KP-th smallest of them bounds the row's KP-th best score from above; it is
+// found by counting (every thread ranks its own minimum among the row's 16).  The few columns at or below that bound
+// (KP of them at least) go to a per-row queue in shared memory, every queued column ranks itself among the row's queue
+// by (score, column) and the first KP write themselves to their place in the list.  A row whose queue overflows (many
+// equal scores, or a tile so narrow that fewer than KP shares hold columns) is scanned again by one thread, column
+// after column.
+// Longer lists (8 or 4 shares): every thread keeps a list over its share, and the shares' lists of a row are merged
+// pairwise, neighbours first, through shared memory, so equal scores keep the order a single scan would give them.
 template <int KP>
-__global__ void __launch_bounds__(2 * kTileM)
-tail_select_kernel(const GemmPlan *__restrict__ plan_dev, int num_ctas, const float *__restrict__ tail_dump,
-                   long long n_entries, float *__restrict__ part_score, int32_t *__restrict__ part_idx) {
-    const GemmPlan plan = *plan_dev;
-    if (plan.mode != 1 || (int)blockIdx.x >= plan.tail_tiles) return;
+struct PieceSplit {
+    static constexpr int value = KP <= 8 ? 16 : KP == 16 ? 8 : 4;
+};
+constexpr int kPieceRowGroups = 2 * kTileM / 32;   // CTAs per tile
+constexpr int kPieceQueue = 64;                    // queued columns per row (short lists)
+
+template <int KP>
+struct PieceSmem {
+    static constexpr int kSplit = PieceSplit<KP>::value;
+    // short lists: the shares' minima and the queues; long lists: the lists on their way through the merge
+    static constexpr int kFloats = KP <= 8 ? kSplit * 32 + 2 * kPieceQueue * 32 : 2 * kSplit * KP * 32;
+};
+
+template <int KP>
+__global__ void __launch_bounds__(32 * PieceSplit<KP>::value, KP <= 8 ? 2 : 1)
+piece_select_kernel(const GemmPlan *__restrict__ plan_dev, int num_ctas, int num_kb, const float *__restrict__ dump,
+                    const float *__restrict__ norms, long long n_entries, float *__restrict__ part_score,
+                    int32_t *__restrict__ part_idx) {
+    constexpr int kSplit = PieceSplit<KP>::value;
     constexpr int kRows = 2 * kTileM;
+    constexpr int kShareCols = kMaxTileN / kSplit;
+    __shared__ float smem_f[PieceSmem<KP>::kFloats];
+    __shared__ int piece_info[4];   // slot of the first piece, slot of the second, CTA of the first, CTA of the last
+    __shared__ int queue_len[32];
+    __shared__ float row_thr[32];
+    const GemmPlan plan = *plan_dev;
+    if (plan.mode != 1 && plan.mode != 3) return;
+    const int lane = threadIdx.x & 31, share = threadIdx.x >> 5;
+    const int rg = blockIdx.x % kPieceRowGroups;
     const long long n16 = (n_entries + 15) / 16;
-    const int id = num_ctas + blockIdx.x;
-    const int n = id / plan.m_tiles, m_tile = id % plan.m_tiles;
-    const long long b0 = n16 * n / plan.n_tiles, b1 = n16 * (n + 1) / plan.n_tiles;
-    const int col0 = (int)(b0 * 16), w = (int)((b1 - b0) * 16);
-    const int row = m_tile * kRows + threadIdx.x;
-    TopList<KP> top;
-    top.reset();
-    const float *base = tail_dump + ((long long)blockIdx.x * plan.tail_slices * kMaxTileN) * kRows + threadIdx.x;
-    for (int c0 = 0; c0 < w; c0 += 16) {
-        float sc[16];
+    const float inf = __int_as_float(0x7F800000);
+    for (int t = blockIdx.x / kPieceRowGroups; t < plan.tail_tiles; t += gridDim.x / kPieceRowGroups) {
+        int n, m_tile;
+        if (plan.mode == 1) {
+            const int id = num_ctas + t;
+            n = id / plan.m_tiles;
+            m_tile = id - n * plan.m_tiles;
+        } else {
+            m_tile = t / plan.n_tiles;
+            n = t - m_tile * plan.n_tiles;
+        }
+        const int rows128 = plan.mode == 3 && plan.half && m_tile == plan.m_tiles - 1 ? 1 : 2;
+        if (rg * 32 >= rows128 * kTileM) continue;   // whole CTA
+        // the pieces of this tile: slot of piece j is j == 0 ? first : second + (j - 1) * stride
+        int stride, pieces;
+        __syncthreads();
+        if (share == 0) {
+            queue_len[lane] = 0;
+            row_thr[lane] = inf;
+        }
+        if (plan.mode == 1) {
+            stride = 1;
+            pieces = plan.tail_slices;
+            if (threadIdx.x == 0) {
+                piece_info[0] = t * plan.tail_slices;
+                piece_info[1] = t * plan.tail_slices + 1;
+            }
+            __syncthreads();
+        } else {
+            // spans are not empty and follow one another: the tile's pieces are those of the query tile's CTAs from
+            // the one whose span holds the tile's first k-block to the one whose span holds its last
+            stride = kMaxSpanItems;
+            int first_cta, cm;
+            span_ctas_of(plan, m_tile, first_cta, cm);
+            const int p_lo = n * num_kb, p_hi = p_lo + num_kb;
+            for (int j = threadIdx.x; j < cm; j += blockDim.x) {
+                const int b0 = span_begin(plan, num_kb, j, cm), b1 = span_begin(plan, num_kb, j + 1, cm);
+                if (b0 <= p_lo && p_lo < b1) {
+                    piece_info[0] = (first_cta + j) * kMaxSpanItems + (n - b0 / num_kb);
+                    piece_info[1] = (first_cta + j + 1) * kMaxSpanItems;
+                    piece_info[2] = j;
+                }
+                if (b0 < p_hi && p_hi <= b1) piece_info[3] = j;
+            }
+            __syncthreads();
+            pieces = piece_info[3] - piece_info[2] + 1;
+        }
+        const int slot0 = piece_info[0], slot1 = piece_info[1];
+        const long long b0 = n16 * n / plan.n_tiles, b1 = n16 * (n + 1) / plan.n_tiles;
+        const int col0 = (int)(b0 * 16), w = (int)((b1 - b0) * 16);
+        const int row_in_tile = rg * 32 + lane;
+        const int row = m_tile * kRows + row_in_tile;
+        const long long out = ((long long)row * plan.lists + n) * KP;
+        auto piece_ptr = [&](int pc, int c0) {
+            return dump + ((long long)(pc == 0 ? slot0 : slot1 + (pc - 1) * stride) * kMaxTileN + c0) * kRows + row_in_tile;
+        };
+        // scores of the 16 columns from c0 on; two pieces' loads in flight, the sums still taken piece after piece
+        auto scores16 = [&](int c0, float (&sc)[16]) {
+            float dot[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) sc[j] = base[(long long)(c0 + j) * kRows];
+            for (int j = 0; j < 16; ++j) dot[j] = 0.f;
+            int pc = 0;
+            for (; pc + 2 <= pieces; pc += 2) {
+                const float *pa = piece_ptr(pc, c0), *pb = piece_ptr(pc + 1, c0);
+                float va[16], vb[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-            if (sc[j] < top.s[KP - 1]) top.insert(sc[j], col0 + c0 + j);
-    }
-    if (row < plan.count) {
-        const long long o = ((long long)row * plan.lists + n) * KP;
+                for (int j = 0; j < 16; ++j) va[j] = __ldg(pa + j * kRows);
 #pragma unroll
-        for (int e = 0; e < KP; ++e) {
-            part_score[o + e] = top.s[e];
-            part_idx[o + e] = top.i[e];
+                for (int j = 0; j < 16; ++j) vb[j] = __ldg(pb + j * kRows);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) dot[j] = (dot[j] + va[j]) + vb[j];
+            }
+            if (pc < pieces) {
+                const float *pa = piece_ptr(pc, c0);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) dot[j] += __ldg(pa + j * kRows);
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int c = col0 + c0 + j;
+                const float nrm = (long long)c < n_entries ? __ldg(norms + c) : inf;
+                sc[j] = fmaf(-2.f, dot[j], nrm);
+            }
+        };
+        if constexpr (KP <= 8) {
+            float *mins = smem_f;                                                  // [share][row]
+            float *queue_s = smem_f + kSplit * 32;                                 // [entry][row]
+            int32_t *queue_i = reinterpret_cast<int32_t *>(queue_s + kPieceQueue * 32);
+            const int c0 = share * 16;
+            float sc[16];
+            float mine = inf;
+            if (c0 < w) {
+                scores16(c0, sc);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) mine = fminf(mine, sc[j]);
+            }
+            mins[share * 32 + lane] = mine;
+            __syncthreads();
+            // rank of this share's minimum among the row's 16 (equal minima: the lower share first)
+            int below = 0;
+#pragma unroll
+            for (int s2 = 0; s2 < kSplit; ++s2) {
+                const float o = mins[s2 * 32 + lane];
+                below += (o < mine || (o == mine && s2 < share)) ? 1 : 0;
+            }
+            if (below == KP - 1) row_thr[lane] = mine;
+            __syncthreads();
+            const float thr = row_thr[lane];
+            if (c0 < w) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    if (sc[j] <= thr && sc[j] < inf) {
+                        const int e = atomicAdd(&queue_len[lane], 1);
+                        if (e < kPieceQueue) {
+                            queue_s[e * 32 + lane] = sc[j];
+                            queue_i[e * 32 + lane] = col0 + c0 + j;
+                        }
+                    }
+                }
+            }
+            __syncthreads();
+            const int queued = queue_len[lane];
+            if (row < plan.count) {
+                if (queued <= kPieceQueue) {
+                    for (int e = share; e < queued; e += kSplit) {
+                        const float ms = queue_s[e * 32 + lane];
+                        const int32_t mi = queue_i[e * 32 + lane];
+                        int rank = 0;
+                        for (int o = 0; o < queued; ++o) {
+                            const float os = queue_s[o * 32 + lane];
+                            rank += (os < ms || (os == ms && queue_i[o * 32 + lane] < mi)) ? 1 : 0;
+                        }
+                        if (rank < KP) {
+                            part_score[out + rank] = ms;
+                            part_idx[out + rank] = mi;
+                        }
+                    }
+                    if (share < KP && share >= queued) {   // fewer columns than list entries
+                        part_score[out + share] = inf;
+                        part_idx[out + share] = -1;
+                    }
+                } else if (share == 0) {
+                    TopList<KP> top;
+                    top.reset();
+                    for (int c1 = 0; c1 < w; c1 += 16) {
+                        float s1[16];
+                        scores16(c1, s1);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (s1[j] < top.s[KP - 1]) top.insert(s1[j], col0 + c1 + j);
+                    }
+#pragma unroll
+                    for (int e = 0; e < KP; ++e) {
+                        part_score[out + e] = top.s[e];
+                        part_idx[out + e] = top.i[e];
+                    }
+                }
+            }
+        } else {
+            float *list_s = smem_f;                                                            // [share][entry][row]
+            int32_t *list_i = reinterpret_cast<int32_t *>(smem_f + kSplit * KP * 32);
+            TopList<KP> top;
+            top.reset();
+            for (int c0 = share * kShareCols; c0 < min(w, (share + 1) * kShareCols); c0 += 16) {
+                float sc[16];
+                scores16(c0, sc);
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (sc[j] < top.s[KP - 1]) top.insert(sc[j], col0 + c0 + j);
+            }
+            // merge neighbours first: the incoming list always holds the higher columns
+            for (int s2 = 1; s2 < kSplit; s2 <<= 1) {
+                if ((share & (2 * s2 - 1)) == s2) {
+#pragma unroll
+                    for (int e = 0; e < KP; ++e) {
+                        list_s[(share * KP + e) * 32 + lane] = top.s[e];
+                        list_i[(share * KP + e) * 32 + lane] = top.i[e];
+                    }
+                }
+                __syncthreads();
+                if ((share & (2 * s2 - 1)) == 0) {
+#pragma unroll
+                    for (int e = 0; e < KP; ++e) {
+                        const float sc = list_s[((share + s2) * KP + e) * 32 + lane];
+                        if (sc < top.s[KP - 1]) top.insert(sc, list_i[((share + s2) * KP + e) * 32 + lane]);
+                    }
+                }
+            }
+            if (share == 0 && row < plan.count) {
+#pragma unroll
+                for (int e = 0; e < KP; ++e) {
+                    part_score[out + e] = top.s[e];
+                    part_idx[out + e] = top.i[e];
+                }
+            }
         }
     }
 }
@@ -1132,16 +1334,12 @@ fi_status_t launch_kp(fi_cache *c, const CUtensorMap &tq, int32_t batch_max, con
     count_launch();
     fi_status_t st = check_launch("gemm_select_kernel");
     if (st != FI_OK || !tail_possible) return st;
-    // the tail kernel reads the plan the GEMM wrote and returns at once when that plan has no tail
-    tail_reduce_kernel<<<dim3(c->sm_count / 2, kMaxTileN / 16), 2 * kTileM, 0, stream>>>(c->plan_dev, c->sm_count, c->tail_dump,
-                                                                                      c->norms, (long long)c->size);
+    // the piece kernel reads the plan the GEMM wrote and returns at once when that plan left no pieces
+    const int num_kb = (c->cfg.dim + kBlockK - 1) / kBlockK;
+    piece_select_kernel<KP><<<kPieceRowGroups * c->sm_count, 32 * PieceSplit<KP>::value, 0, stream>>>(
+        c->plan_dev, c->sm_count, num_kb, c->tail_dump, c->norms, (long long)c->size, c->part_score, c->part_idx);
     count_launch();
-    st = check_launch("tail_reduce_kernel");
-    if (st != FI_OK) return st;
-    tail_select_kernel<KP><<<c->sm_count / 2, 2 * kTileM, 0, stream>>>(c->plan_dev, c->sm_count, c->tail_dump,
-                                                                       (long long)c->size, c->part_score, c->part_idx);
-    count_launch();
-    return check_launch("tail_select_kernel");
+    return check_launch("piece_select_kernel");
 }
 
 // The pair kernel: clusters of two CTAs, one pair per two SMs.
@@ -1273,14 +1471,14 @@ size_t gemm_part_entries(int max_batch, int64_t capacity, int sm_count, int k, i
 
 size_t gemm_part_entries_bound(int max_batch, int64_t capacity, int sm_count, int k, int dim) {
     // lists per query: at most one per range (ranges <= CTAs, and <= 16-row blocks of the cache), times two for
-    // 128-row tiles (two epilogue warps per row); wave + tail mode has one list per 256-row tile of the cache,
-    // at most 1.5 x CTAs of them
+    // 128-row tiles (two epilogue warps per row); wave + tail and spans modes have one list per 256-row tile of the
+    // cache, at most 1.5 x CTAs and 2 x CTAs of them
     const size_t n16 = (size_t)((capacity + 15) / 16);
     const size_t list_len = (size_t)gemm_list_len(k);
     auto entries = [&](int rows, int tile_m) {
         const size_t f = tile_m == kTileM ? 2 : 1;
         size_t lists = (size_t)sm_count * f;
-        if (tile_m != kTileM && lists < (size_t)sm_count + sm_count / 2) lists = (size_t)sm_count + sm_count / 2;
+        if (tile_m != kTileM && lists < (size_t)2 * sm_count) lists = (size_t)2 * sm_count;
         if (lists > n16 * f) lists = n16 * f;
         if (lists < f) lists = f;
         const size_t padded = (size_t)((rows + tile_m - 1) / tile_m) * tile_m;
@@ -1294,18 +1492,21 @@ size_t gemm_part_entries_bound(int max_batch, int64_t capacity, int sm_count, in
     return worst;
 }
 
+// slots of 256 x 256 partial sums: one per CTA in wave + tail mode, kMaxSpanItems per CTA in spans mode
 size_t gemm_tail_units(int max_batch, int dim, int sm_count) {
     const int num_kb = (dim + kBlockK - 1) / kBlockK;
-    return gemm_tile_m(max_batch, dim) == 2 * kTileM && num_kb >= 64 ? (size_t)sm_count : 0;
+    return gemm_tile_m(max_batch, dim) == 2 * kTileM && num_kb >= 64 ? (size_t)sm_count * kMaxSpanItems : 0;
 }
 
-// Can a batch of at most batch_max requests against the current cache end up in wave + tail mode?
+// Can a batch of at most batch_max requests against the current cache end up in a mode that leaves pieces (wave +
+// tail, spans)?  The mode depends on the number of query tiles and on whether the last one is at most half full.
 static bool tail_mode_possible(const fi_cache *c, int batch_max) {
     const int tile_m = gemm_tile_m(batch_max, c->cfg.dim);
     const int num_kb = (c->cfg.dim + kBlockK - 1) / kBlockK;
     const int m_tiles_max = (batch_max + tile_m - 1) / tile_m;
     for (int mt = 1; mt <= m_tiles_max; ++mt)
-        if (make_gemm_plan(mt * tile_m, c->size, c->sm_count, c->cfg.k, tile_m, num_kb).mode == 1) return true;
+        for (int count : {mt * tile_m, mt * tile_m - tile_m / 2})
+            if (make_gemm_plan(count, c->size, c->sm_count, c->cfg.k, tile_m, num_kb).mode != 0) return true;
     return false;
 }
 
@@ -1346,9 +1547,10 @@ fi_status_t launch_gemm_select(fi_cache *c, const void *queries_compact, int64_t
     st = encode_bf16_map(&tq, queries_compact, (uint64_t)batch_max, (uint64_t)c->cfg.dim, (uint64_t)ld_elems, kTileM);
     if (st != FI_OK) return st;
     const bool tail_possible = tail_mode_possible(c, batch_max);
-    if (tail_possible && c->tail_dump_units < (size_t)c->sm_count) {
-        // one slot of 256 x 256 partial sums per CTA, allocated at create for every cache whose shapes can get here
-        set_error("the distance GEMM's partial-sum buffer is missing (%zu slots, %d needed)", c->tail_dump_units, c->sm_count);
+    if (tail_possible && c->tail_dump_units < (size_t)c->sm_count * kMaxSpanItems) {
+        // slots of 256 x 256 partial sums, allocated at create for every cache whose shapes can get here
+        set_error("the distance GEMM's partial-sum buffer is missing (%zu slots, %d needed)", c->tail_dump_units,
+                  c->sm_count * kMaxSpanItems);
         return FI_ERR_CAPACITY;
     }
     if (use_pair_kernel(c, batch_max)) return launch_pair<1>(c, tq, batch_max, count_dev, stream);

@@ -38,6 +38,16 @@ __host__ __device__ inline int gemm_list_len(int k) {
 // then gives each CTA one full tile over the whole row length, and the tiles left over are cut along the row
 // length into `tail_slices` pieces, one per CTA; their partial sums go to memory and a small kernel adds them
 // up and selects.
+//
+// When there is less than one 256 x 256 tile per CTA ("spans" mode), ranges would be narrow tiles under a query tile
+// that every CTA reads in full.  Instead every query tile gets an equal share of the CTAs, and the (cache-row tile,
+// k-block) pairs of that query tile, laid end to end, are cut into one span per CTA of its share: a CTA runs the
+// k-blocks of its span (the end of one tile and the start of the next, at most kMaxSpanItems pieces), every piece
+// leaves its partial sums in memory, and the same small kernel adds up the pieces of each tile and selects.  The
+// spans of all query tiles have the same boundaries, so the CTAs that need the same cache rows read them at the same
+// time; the query tiles are read at scattered times and have to stay in L2, which bounds their size.  A last query
+// tile with at most 128 requests computes half (one of its two 128-row MMAs) and gets 3/4 of a share: its k-blocks
+// still load the full cache-row tile.
 struct GemmPlan {
     int32_t count;        // actual batch
     int32_t m_tiles;      // ceil(count / tile_m)
@@ -48,12 +58,43 @@ struct GemmPlan {
     int32_t list_len;     // entries per candidate list
     int32_t tile_m;       // query rows per CTA tile
     int32_t lists;        // candidate lists per query
-    int32_t mode;         // 0 = ranges, 1 = wave + tail, 2 = pieces only (plain product, no select)
-    int32_t n_tiles;      // wave + tail, pieces: cache-row tiles per query tile
-    int32_t tail_tiles;   // wave + tail: tiles beyond the first wave; pieces: all tiles
+    int32_t mode;         // 0 = ranges, 1 = wave + tail, 2 = pieces only (plain product, no select), 3 = spans
+    int32_t n_tiles;      // wave + tail, pieces, spans: cache-row tiles per query tile
+    int32_t tail_tiles;   // wave + tail: tiles beyond the first wave; pieces, spans: all tiles
     int32_t tail_slices;  // wave + tail, pieces: pieces each of those tiles is cut into along the row length
     int32_t pieces;       // pieces: tail_tiles * tail_slices
+    int32_t half;         // spans: 1 = the last query tile holds at most 128 requests
+    int32_t span_full;    // spans: CTAs per full query tile
+    int32_t span_half;    // spans: CTAs of the half query tile
 };
+
+constexpr int kMaxSpanItems = 3;   // pieces a span can consist of (spans are at most two tiles' k-blocks long)
+constexpr int kMinSpanKb = 16;     // shortest span worth a CTA, in k-blocks
+
+// Spans mode: which query tile CTA `cta` works for, its index among that tile's CTAs and their number (false: idle)
+__host__ __device__ inline bool span_owner(const GemmPlan &p, int cta, int &m, int &j, int &cm) {
+    const int mf = p.m_tiles - p.half, full_ctas = mf * p.span_full;
+    if (cta < full_ctas) {
+        m = cta / p.span_full;
+        j = cta - m * p.span_full;
+        cm = p.span_full;
+        return true;
+    }
+    m = p.m_tiles - 1;
+    j = cta - full_ctas;
+    cm = p.span_half;
+    return j < p.half * p.span_half;
+}
+// first CTA and number of CTAs of query tile m
+__host__ __device__ inline void span_ctas_of(const GemmPlan &p, int m, int &first, int &cm) {
+    const int mf = p.m_tiles - p.half;
+    first = m < mf ? m * p.span_full : mf * p.span_full;
+    cm = m < mf ? p.span_full : p.span_half;
+}
+// position, in (cache-row tile, k-block) pairs of one query tile, where the j-th of cm spans starts (j = cm: the end)
+__host__ __device__ inline int span_begin(const GemmPlan &p, int num_kb, int j, int cm) {
+    return j * (p.n_tiles * num_kb) / cm;
+}
 
 // `pair`: the workers are pairs of CTAs that share one tile of tile_m rows (half each; pair_lists epilogue warps, hence
 // lists, per row; ranges only, range lengths a multiple of 32 rows); num_ctas is then the number of pairs.
@@ -68,6 +109,7 @@ __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entrie
     p.lists = 0;
     p.mode = 0;
     p.n_tiles = p.tail_tiles = p.tail_slices = 0;
+    p.half = p.span_full = p.span_half = 0;
     long long n16 = (n_entries + 15) / 16;
     if (p.m_tiles <= 0 || n16 <= 0) {
         p.mg = p.groups = p.parts = 1;
@@ -78,6 +120,37 @@ __host__ __device__ inline GemmPlan make_gemm_plan(int count, long long n_entrie
     if (tile_m == 2 * kTileM && num_kb >= 64 && !pair) {
         const long long nt = (n16 + 15) / 16;                 // tiles of at most 256 rows
         const long long total = (long long)p.m_tiles * nt;
+        // Spans: less than a tile per CTA (a half tile counts 3/4: half the MMAs, 3/4 of the operand bytes), query
+        // tiles of at most 16 MB together, and 32-bit span arithmetic.
+        const int half = count - (p.m_tiles - 1) * tile_m <= kTileM ? 1 : 0;
+        const int mf = p.m_tiles - half;
+        if ((4 * mf + 3 * half) * nt <= 4 * num_ctas && (long long)p.m_tiles * num_kb <= 512 &&
+            (long long)num_ctas * nt * num_kb < 2147483647ll) {
+            const int len = (int)nt * num_kb;                       // pairs per query tile
+            const int cap = len / kMinSpanKb > 0 ? len / kMinSpanKb : 1;
+            int ch = half ? (mf ? num_ctas * 3 / (4 * mf + 3) : num_ctas) : 0;
+            if (half && ch < 1) ch = 1;
+            int cf = mf ? (num_ctas - ch) / mf : 0;
+            if (ch > cap) ch = cap;
+            if (cf > cap) cf = cap;
+            // the longest span (len / c rounded up) may touch kMaxSpanItems tiles at most
+            const bool fits = (!mf || (cf >= 1 && (len + cf - 1) / cf <= 2 * num_kb)) &&
+                              (!half || (len + ch - 1) / ch <= 2 * num_kb);
+            if (fits) {
+                p.mode = 3;
+                p.n_tiles = (int32_t)nt;
+                p.tail_tiles = (int32_t)total;
+                p.half = half;
+                p.span_full = cf;
+                p.span_half = ch;
+                p.mg = p.m_tiles;
+                p.groups = 1;
+                p.parts = (int32_t)nt;
+                p.range16 = 16;
+                p.lists = (int32_t)nt;
+                return p;
+            }
+        }
         if (total > num_ctas && total <= num_ctas + num_ctas / 2) {
             p.mode = 1;
             p.n_tiles = (int32_t)nt;

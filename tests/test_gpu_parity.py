@@ -104,6 +104,10 @@ def test_stream_path_large_dim_reads_queries_in_place():
     (9000, 320, 2048, 1),      # the same with list length 4, K = 5 blocks
     (33000, 1024, 1100, 5),    # rows of 1,024 values, many entries, batch above 1,024: pairs of CTAs share 256-row tiles
     (40001, 2048, 1024, 10),   # the same with list length 16, ragged entry count, 4 query tiles of a pair exactly
+    (9990, 4096, 803, 5),      # deep rows, fewer tiles than CTAs once the last query tile (35 requests) counts half: spans
+    (2500, 8192, 190, 5),      # one query tile x 10 cache tiles over 148 CTAs: about 15 pieces per tile
+    (7000, 4096, 482, 13),     # two query tiles, list length 16, spans that cross from one tile into the next
+    (300, 4096, 200, 29),      # two ragged cache tiles, list length 32, fewer spans than CTAs
 ])
 def test_gemm_path(n, d, b, k):
     w = dg.single_layer(name="t", n_cache=n, n_query=b, dim=d, num_classes=9, dtype="bf16", sigma=0.6, k=k, seed=5)
@@ -314,6 +318,15 @@ def test_cascade_resnet18_shape_shrunk(path):
 
 def test_cascade_imagenet_shape_shrunk():
     check_cascade(dg.config4(seed=0, shrink=8), fb.FI_PATH_GEMM)
+
+
+def test_cascade_of_deep_rows_whose_batch_shrinks_below_half_a_tile():
+    # 600 requests (three 256-row tiles, the last at most half full at some stage) down to fewer than 128 (one half
+    # tile) against rows of 4,096 values: every stage runs the spans form of the distance GEMM
+    w = dg.cascade(name="t", dims=[4096, 4096, 4096, 4096], scales=[0.2, 0.4, 0.8, 1.6], kind="halfnormal", n_cache=1500,
+                   n_query=600, n_calib=128, num_classes=10, dtype="bf16", k=5, seed=5)
+    w.meta.update(rule="conf_gt", percentiles=[45.0, 40.0, 40.0, 40.0])
+    check_cascade(w, fb.FI_PATH_GEMM)
 
 
 def test_cascade_threshold_limits():
