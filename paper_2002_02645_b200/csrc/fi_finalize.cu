@@ -285,10 +285,10 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
         cand_w[tid] = p.weights[cand_i[tid]];
     }
     // ---- exact distances of the candidates.  The row length is cut into blocks of 32 chunks of 16 bytes; warp w takes
-    // every kFinWarps-th block and, for its blocks, reads the query ONCE and up to eight candidate rows against it
-    // (nine 16-byte loads in flight per lane).  A warp per candidate, each walking the whole query, read the query
-    // eight times over and was bound by the traffic from L2 to the SMs on long rows (2.2 GB for 1,024 requests of
-    // 65,536 values, of which the candidates are 1.07 GB) and by a chain of dependent DRAM round trips on small batches.
+    // every kFinWarps-th block and, for its blocks, reads the query once and up to eight candidate rows against it
+    // (nine 16-byte loads in flight per lane).  A warp per candidate, each walking the whole row with four loads in
+    // flight, was bound by the latency of its 32 dependent iterations.  (The packed fp32 subtract and multiply-add of
+    // this architecture, two elements per instruction, were measured here too: slower, and 16 more registers.)
     // The partial sums are added in a fixed order (lanes by shuffle tree, then warps 0..7), so reruns are bit-identical.
     if (p.refine) {
         constexpr int kGroup = 8;   // candidates per pass over the query

@@ -1016,7 +1016,7 @@ piece_select_kernel(const GemmPlan *__restrict__ plan_dev, int num_ctas, int num
             n = t - m_tile * plan.n_tiles;
         }
         const int rows128 = plan.mode == 3 && plan.half && m_tile == plan.m_tiles - 1 ? 1 : 2;
-        if (rg * 32 >= rows128 * kTileM) continue;   // whole CTA
+        if (rg * 32 >= rows128 * kTileM || m_tile * kRows + rg * 32 >= plan.count) continue;   // whole CTA: no request here
         // the pieces of this tile: slot of piece j is j == 0 ? first : second + (j - 1) * stride
         int stride, pieces;
         __syncthreads();
