@@ -341,6 +341,20 @@ fi_status_t fi_cache_read_slot_certificates(fi_cache_t *cache, uint8_t *flags_ho
 fi_status_t fi_cache_set_profiling(fi_cache_t *cache, int32_t enable);
 fi_status_t fi_cache_read_profile(fi_cache_t *cache, float *total_ms, int32_t *launches);
 
+/* Host only (no GPU call): how the distance GEMM of a look-up of `count` requests (in a call sized for `max_batch`)
+ * against `n_entries` bf16 entries of `dim` values would be split over `num_ctas` CTAs.
+ * plan_out[0..16] = count, query tiles, tiles per group, groups, cache-row ranges, rows per range / 16, list length,
+ * rows per query tile, lists per query, mode (0 ranges, 1 wave + tail, 3 spans), cache-row tiles per query tile,
+ * tiles left in pieces, pieces per tail tile, 0, half-full last query tile (0 / 1), CTAs per full query tile, CTAs
+ * of the half-full one (the last three: spans mode).
+ * If `cta` >= 0 and the mode is spans, items_out receives that CTA's pieces, six values each (query tile, cache-row
+ * tile, first k-block, end k-block, 128-row MMAs, slot of the partial sums), and *n_items their number (at most 3);
+ * in other modes *n_items = 0.  plan_out, items_out (18 values) and n_items are host pointers owned by the caller.
+ * Errors: FI_ERR_INVALID_ARG for null plan_out or non-positive sizes.  Used by the tests of the host logic. */
+fi_status_t fi_gemm_plan_describe(int32_t count, int64_t n_entries, int32_t num_ctas, int32_t k, int32_t dim,
+                                  int32_t max_batch, int32_t cta, int32_t *plan_out, int32_t *items_out,
+                                  int32_t *n_items);
+
 /* Number of kernels this library has launched in the calling process (all caches). */
 int64_t fi_launch_count(void);
 

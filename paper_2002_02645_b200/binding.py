@@ -28,7 +28,7 @@ EXPORTS = ["fi_cache_create", "fi_cache_destroy", "fi_cache_insert", "fi_cache_s
            "fi_projection_create", "fi_projection_destroy", "fi_projection_set_weights", "fi_projection_apply", "fi_projection_poll_status", "fi_projection_set_profiling",
            "fi_projection_read_profile",
            "fi_cascade_step_projected", "fi_cache_set_repair", "fi_cache_read_certificate",
-           "fi_cache_read_slot_certificates", "fi_cache_lookup_view", "fi_cache_set_sm_limit", "fi_launch_count", "fi_last_error", "fi_status_string"]
+           "fi_cache_read_slot_certificates", "fi_cache_lookup_view", "fi_cache_set_sm_limit", "fi_gemm_plan_describe", "fi_launch_count", "fi_last_error", "fi_status_string"]
 
 
 class fi_cache_config_t(ctypes.Structure):
@@ -107,6 +107,9 @@ def load_library(path: Optional[str] = None):
     lib.fi_cache_read_slot_certificates.argtypes = [vp, vp, i32]
     lib.fi_cache_set_profiling.argtypes = [vp, i32]
     lib.fi_cache_read_profile.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
+    lib.fi_gemm_plan_describe.argtypes = [i32, i64, i32, i32, i32, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                          ctypes.POINTER(i32)]
+    lib.fi_gemm_plan_describe.restype = i32
     lib.fi_launch_count.argtypes = []
     lib.fi_launch_count.restype = i64
     lib.fi_last_error.argtypes = []
@@ -128,6 +131,21 @@ def status_string(status: int) -> str:
 def _check(status: int) -> None:
     if status != FI_OK:
         raise FiError(status, load_library().fi_last_error().decode())
+
+
+PLAN_FIELDS = ("count", "m_tiles", "mg", "groups", "parts", "range16", "list_len", "tile_m", "lists", "mode", "n_tiles",
+               "tail_tiles", "tail_slices", "pieces", "half", "span_full", "span_half")
+
+
+def gemm_plan_describe(count: int, n_entries: int, num_ctas: int, k: int, dim: int, max_batch: int, cta: int = -1):
+    """Host only: the work split of the distance GEMM as a dict, plus (spans mode, cta >= 0) that CTA's pieces as
+    tuples (query tile, cache-row tile, first k-block, end k-block, 128-row MMAs, slot)."""
+    plan = (ctypes.c_int32 * 17)()
+    items = (ctypes.c_int32 * 18)()
+    n = ctypes.c_int32(0)
+    _check(load_library().fi_gemm_plan_describe(count, n_entries, num_ctas, k, dim, max_batch, cta, plan, items,
+                                                ctypes.byref(n)))
+    return dict(zip(PLAN_FIELDS, plan)), [tuple(items[6 * i:6 * i + 6]) for i in range(n.value)]
 
 
 def launch_count() -> int:

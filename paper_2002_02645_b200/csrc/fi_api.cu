@@ -1155,6 +1155,39 @@ fi_status_t fi_cache_read_slot_certificates(fi_cache_t *c, uint8_t *flags_host, 
     return FI_OK;
 }
 
+fi_status_t fi_gemm_plan_describe(int32_t count, int64_t n_entries, int32_t num_ctas, int32_t k, int32_t dim,
+                                  int32_t max_batch, int32_t cta, int32_t *plan_out, int32_t *items_out,
+                                  int32_t *n_items) {
+    if (!plan_out || count <= 0 || n_entries <= 0 || num_ctas <= 0 || k <= 0 || dim <= 0 || max_batch < count) {
+        set_error("fi_gemm_plan_describe: null or non-positive argument");
+        return FI_ERR_INVALID_ARG;
+    }
+    const int tile_m = gemm_tile_m(max_batch, dim);
+    const int num_kb = (dim + 63) / 64;
+    const GemmPlan p = make_gemm_plan(count, n_entries, num_ctas, k, tile_m, num_kb);
+    const int32_t v[17] = {p.count, p.m_tiles, p.mg, p.groups, p.parts, p.range16, p.list_len, p.tile_m, p.lists, p.mode,
+                           p.n_tiles, p.tail_tiles, p.tail_slices, p.pieces, p.half, p.span_full, p.span_half};
+    for (int i = 0; i < 17; ++i) plan_out[i] = v[i];
+    if (n_items) *n_items = 0;
+    int m, j, cm;
+    if (p.mode == 3 && cta >= 0 && items_out && n_items && span_owner(p, cta, m, j, cm)) {
+        const int s0 = span_begin(p, num_kb, j, cm), s1 = span_begin(p, num_kb, j + 1, cm);
+        const int n = s1 > s0 ? (s1 - 1) / num_kb - s0 / num_kb + 1 : 0;
+        for (int idx = 0; idx < n && idx < kMaxSpanItems; ++idx) {
+            const int tile = s0 / num_kb + idx;
+            int32_t *it = items_out + 6 * idx;
+            it[0] = m;
+            it[1] = tile;
+            it[2] = idx == 0 ? s0 - tile * num_kb : 0;
+            it[3] = s1 - tile * num_kb < num_kb ? s1 - tile * num_kb : num_kb;
+            it[4] = p.half && m == p.m_tiles - 1 ? 1 : 2;
+            it[5] = cta * kMaxSpanItems + idx;
+        }
+        *n_items = n;
+    }
+    return FI_OK;
+}
+
 int64_t fi_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
 
 const char *fi_last_error(void) { return g_err; }

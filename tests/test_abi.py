@@ -83,3 +83,55 @@ def test_gemm_plan_is_balanced():
         assert (parts - 1) * r16 * 16 < n <= parts * r16 * 16
         ideal = (-(-count // 128)) * (-(-n // 16)) / 148
         assert groups * r16 <= max(1.35 * ideal, ideal + groups)      # within 35 % of a perfect split
+
+
+def test_spans_partition_every_tile_exactly_once():
+    """Spans mode of the distance GEMM, from the library's own plan code (host only): for every query tile the pieces
+    of all CTAs cover each (cache-row tile, k-block) pair exactly once, a CTA has at most three pieces, slots are
+    distinct, and the half-full last query tile takes one 128-row MMA."""
+    from paper_2002_02645_b200 import binding as fb
+    cases = [  # count, entries, dim, max_batch
+        (190, 10000, 8192, 1024), (482, 10000, 16384, 1024), (100, 10000, 8192, 1024), (300, 3000, 4096, 600),
+        (270, 1500, 4096, 600), (200, 300, 4096, 200), (129, 16, 4096, 129), (600, 1500, 4096, 600), (35, 700, 65536, 1024)]
+    seen_modes = set()
+    for count, n, dim, max_batch in cases:
+        plan, _ = fb.gemm_plan_describe(count, n, 148, 5, dim, max_batch)
+        seen_modes.add(plan["mode"])
+        if plan["mode"] != 3:
+            continue
+        num_kb = (dim + 63) // 64
+        covered = {}
+        slots = set()
+        for cta in range(148):
+            _, items = fb.gemm_plan_describe(count, n, 148, 5, dim, max_batch, cta)
+            assert len(items) <= 3
+            for m, tile, kb0, kb1, rows128, slot in items:
+                assert 0 <= kb0 < kb1 <= num_kb and 0 <= tile < plan["n_tiles"] and 0 <= m < plan["m_tiles"]
+                assert rows128 == (1 if plan["half"] and m == plan["m_tiles"] - 1 else 2)
+                assert slot not in slots and slot // 3 == cta
+                slots.add(slot)
+                for kb in range(kb0, kb1):
+                    assert (m, tile, kb) not in covered
+                    covered[(m, tile, kb)] = cta
+        assert len(covered) == plan["m_tiles"] * plan["n_tiles"] * num_kb
+        # the pieces of one tile come from consecutive CTAs, in k order
+        for m in range(plan["m_tiles"]):
+            for tile in range(plan["n_tiles"]):
+                owners = [covered[(m, tile, kb)] for kb in range(num_kb)]
+                assert owners == sorted(owners) and set(owners) == set(range(owners[0], owners[-1] + 1))
+        assert plan["lists"] == plan["n_tiles"] and plan["half"] == (1 if count - (plan["m_tiles"] - 1) * 256 <= 128 else 0)
+    assert 3 in seen_modes
+
+
+def test_plan_modes_of_the_bench_workloads():
+    from paper_2002_02645_b200 import binding as fb
+    mode = lambda count, n, dim, mb, k=5: fb.gemm_plan_describe(count, n, 148, k, dim, mb)[0]["mode"]
+    assert mode(1024, 10000, 65536, 1024) == 1      # one full tile per CTA and a tail cut along the rows
+    assert mode(803, 10000, 32768, 1024) == 1
+    assert mode(482, 10000, 16384, 1024) == 3       # fewer tiles than CTAs: spans
+    assert mode(190, 10000, 8192, 1024) == 3
+    assert mode(8192, 200000, 8192, 8192, 10) == 0  # many tiles per CTA: ranges
+    assert mode(4096, 100000, 256, 4096) == 0
+    p, _ = fb.gemm_plan_describe(8192, 200000, 148, 10, 8192, 8192)
+    assert p["mg"] * 256 * 8192 * 2 <= 48 << 20     # a group's query tiles stay under 48 MB over a cache beyond L2
+    assert fb.load_library().fi_gemm_plan_describe(0, 10, 148, 5, 64, 16, -1, None, None, None) == 1
