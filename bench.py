@@ -448,8 +448,8 @@ def measure_ours(args, workload, batch, *, full=True):
         flops = 2.0 * b0 * n0 * d0
         nbytes = n0 * d0 * st0.cache_vecs.itemsize + b0 * d0 * st0.cache_vecs.itemsize + 4.0 * n0
         gemm = st0.dtype == "bf16" and b0 > 1      # the library's own rule: single requests and fp32 caches stream
-        # the events bracket the distance kernel of a look-up: gemm_select_kernel (followed, in wave + tail mode, by
-        # its two small tail kernels) or stream_lookup_kernel
+        # the events bracket the distance kernel of a look-up: gemm_select_kernel (followed, where tiles were cut along the row length, by
+        # piece_select_kernel) or stream_lookup_kernel
         kernel = "gemm_select_kernel" if gemm else "stream_lookup_kernel"
         # the slower of the flops at the tensor peak and the bytes at the copy bandwidth bounds the launch
         tensor_bound = gemm and flops / (peaks["bf16_tflops"] * 1e12) > nbytes / (peaks["hbm_gbs"] * 1e9)
