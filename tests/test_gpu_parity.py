@@ -114,6 +114,30 @@ def test_gemm_path(n, d, b, k):
     check_case(w.stages[0], k=k, num_classes=9, rule=fo.RULE_CONF_GT, path=fb.FI_PATH_GEMM)
 
 
+@pytest.mark.parametrize("n,d,b,first", [
+    (600, 4096, 200, 100),      # spans: three cache tiles, the duplicates inside the first and second
+    (9990, 4096, 900, 9500),    # wave + tail: the duplicates sit in tiles that are cut along the row length
+    (40000, 256, 300, 7000),    # ranges with the select in the GEMM's epilogue
+])
+def test_many_equal_scores_keep_the_lowest_indices(n, d, b, first):
+    """150 identical cache rows nearer to every query than anything else: every list, queue and merge on the way sees
+    150 equal scores and must keep those with the lowest indices, as the oracle's (distance, index) order does."""
+    k = 5
+    w = dg.single_layer(name="t", n_cache=n, n_query=b, dim=d, num_classes=1, dtype="bf16", sigma=0.6, k=k, seed=11)
+    st = w.stages[0]
+    # one class: the mean of the queries (rounded to bf16) is nearer to each of them than an independent row is
+    mean = torch.from_numpy(st.queries.view(np.int16).copy()).view(torch.bfloat16).float().mean(0).to(torch.bfloat16)
+    st.cache_vecs[first:first + 150] = mean.view(torch.int16).numpy().view(np.uint16)[None, :]
+    ref = fo.lookup(st.queries[:8], st.cache_vecs, st.cache_labels, k=k, tau=0.0)
+    np.testing.assert_array_equal(ref.ni, np.tile(np.arange(first, first + k), (8, 1)))   # the premise, by the oracle
+    cache = make_cache(st, k=k, num_classes=1, tau=0.0, max_batch=b, path=fb.FI_PATH_GEMM)
+    got = run_lookup(cache, st.queries)
+    np.testing.assert_array_equal(got[4], np.tile(np.arange(first, first + k, dtype=np.int32), (b, 1)))
+    assert (got[3] == got[3][:, :1]).all()
+    np.testing.assert_allclose(got[3][:8], ref.nd, rtol=2e-3)
+    cache.close()
+
+
 def test_gemm_and_stream_paths_agree_and_copies_hit():
     w = dg.single_layer(name="t", n_cache=3000, n_query=40, dim=512, num_classes=6, dtype="bf16", sigma=0.5, k=5,
                         seed=6, n_copies=8)
