@@ -95,7 +95,9 @@ typedef struct {
 
 /*
  * Create the (empty) cache of one layer: CACHE[layer] = {} and THRESHOLDS[layer] of Pseudocode 1.
- * Allocates capacity*dim elements plus labels, weights, norms and look-up scratch on cfg->device.
+ * Allocates capacity*dim elements plus labels, weights, norms and look-up scratch on cfg->device (the scratch:
+ * candidate lists for max_batch requests, and for bf16 rows of 4,096 values and more under batches above 128 also
+ * three 256 KiB slots of partial sums per SM, about 116 MB).
  * Synchronous.  Errors: INVALID_ARG (null, dim/k/capacity/max_batch out of range, dim not a multiple
  * of 8 (bf16) or 4 (f32)), OOM, CUDA.  On error *out is NULL.
  */
