@@ -138,6 +138,48 @@ def test_many_equal_scores_keep_the_lowest_indices(n, d, b, first):
     cache.close()
 
 
+def test_tensor_core_and_streaming_paths_agree_on_random_deep_shapes():
+    """Consistency, not parity (no oracle here): on 16 seeded random shapes of deep rows (4,096-16,384 values, 129-900
+    requests behind a gather list, a device-resident count, sometimes an SM limit) the tensor-core path, whose work split
+    changes form with every one of these numbers, returns the neighbours and distances of the streaming path, which
+    computes every distance directly.  A differing neighbour set is accepted only for a tie at the k-th place."""
+    rng = np.random.default_rng(7)
+    forms = set()
+    fixed = [(8192, 800, 11700, 13, 800, 0), (16384, 600, 20, 5, 600, 0)]   # wave + tail; ranges over a handful of rows
+    for case in range(16):
+        d = int(rng.choice([4096, 4160, 8192, 16384]))
+        b = int(rng.integers(129, 900))
+        n = int(rng.choice([rng.integers(1, 40), rng.integers(40, 600), rng.integers(600, 12000)]))
+        k = int(rng.choice([1, 5, 13, 29]))
+        count = int(rng.integers(1, b + 1)) if rng.random() < 0.6 else b
+        sms = int(rng.choice([0, 0, 100, 37, 8]))
+        if case < len(fixed):
+            d, b, n, k, count, sms = fixed[case]
+        w = dg.single_layer(name="f", n_cache=n, n_query=b, dim=d, num_classes=7, dtype="bf16", sigma=0.6, k=k,
+                            seed=int(rng.integers(1 << 30)))
+        st = w.stages[0]
+        forms.add(fb.gemm_plan_describe(count, n, sms or 148, k, d, b)[0]["mode"])
+        perm = torch.from_numpy(rng.permutation(b).astype(np.int32)).to("cuda:0")
+        cnt = torch.tensor([count], dtype=torch.int32, device="cuda:0")
+        res = []
+        for path in (fb.FI_PATH_STREAM, fb.FI_PATH_GEMM):
+            c = make_cache(st, k=k, num_classes=7, tau=0.0, max_batch=b + 100, path=path)
+            if sms:
+                c.set_sm_limit(sms)
+            out = c.lookup_batch(to_device(st.queries), row_idx=perm, batch_max=b, batch_count=cnt)
+            torch.cuda.synchronize()
+            c.poll_status()
+            res.append((out.topk_dist.cpu().numpy()[:count], out.topk_idx.cpu().numpy()[:count]))
+            c.close()
+        (d0, i0), (d1, i1) = res
+        ke = min(k, n)
+        np.testing.assert_allclose(d1[:, :ke], d0[:, :ke], rtol=2e-3)
+        for r in range(count):
+            if set(i0[r, :ke]) != set(i1[r, :ke]):
+                assert abs(d0[r, ke - 1] - d1[r, ke - 1]) <= 1e-4 * d0[r, ke - 1], (d, b, n, k, count, sms, r)
+    assert forms == {0, 1, 3}
+
+
 def test_gemm_and_stream_paths_agree_and_copies_hit():
     w = dg.single_layer(name="t", n_cache=3000, n_query=40, dim=512, num_classes=6, dtype="bf16", sigma=0.5, k=5,
                         seed=6, n_copies=8)
