@@ -14,6 +14,9 @@ constexpr int kStreamThreads = 256;
 constexpr int kStreamWarps = kStreamThreads / 32;
 constexpr int kRowsPerIter = 4;   // cache rows in flight per thread: 4 x 16 B loads
 constexpr int kQB = 4;            // queries served by one pass over the rows
+// A single request leaves the registers of three more accumulators per row free: eight rows in flight per thread
+// instead of four, which is what the memory system needs from 768 threads per SM to run at its full rate.
+constexpr int kRowsPerIterSingle = 8;
 
 __device__ __forceinline__ uint4 ld_stream16(const void *p) {
     uint4 v;
@@ -114,29 +117,29 @@ __global__ void gather_rows_kernel(const char *__restrict__ src, int64_t ld_byte
 }
 
 // ---------------------------------------------------------------- K5: streaming look-up
-// grid = (parts, ceil(batch_max / 4)); CTA (p, g) scans the p-th range of cache rows for queries 4g..4g+3 and
-// writes one sorted list of the k best (distance, index) pairs per query.
-template <typename T>
+// grid = (parts, ceil(batch_max / QB)); CTA (p, g) scans the p-th range of cache rows for queries QB*g..QB*g+QB-1 and
+// writes one sorted list of the k best (distance, index) pairs per query.  (QB, ROWS) = (4, 4), or (1, 8) for one request.
+template <typename T, int QB, int ROWS>
 __global__ void __launch_bounds__(kStreamThreads)
 stream_lookup_kernel(const T *__restrict__ X, int64_t n_entries, int dim, const T *__restrict__ Q, int64_t ldq,
                      const int32_t *__restrict__ row_idx, int32_t batch_max, const int32_t *__restrict__ count_dev,
                      int k, int parts, int q_in_smem, float *__restrict__ part_score, int32_t *__restrict__ part_idx) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ float red[kStreamWarps][kRowsPerIter * kQB];
-    __shared__ float best_d[kQB][kMaxK];
-    __shared__ int32_t best_i[kQB][kMaxK];
+    __shared__ float red[kStreamWarps][ROWS * QB];
+    __shared__ float best_d[QB][kMaxK];
+    __shared__ int32_t best_i[QB][kMaxK];
 
     const int count = count_dev ? min(*count_dev, batch_max) : batch_max;
-    const int q0 = blockIdx.y * kQB;
+    const int q0 = blockIdx.y * QB;
     if (q0 >= count) return;
-    const int nq = min(kQB, count - q0);
+    const int nq = min(QB, count - q0);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chunks = dim / Elem<T>::kPer16;
 
     // query rows: in shared memory when they fit, else read in place (they stay in L1/L2)
-    const uint4 *qrow[kQB];
+    const uint4 *qrow[QB];
 #pragma unroll
-    for (int j = 0; j < kQB; ++j) {
+    for (int j = 0; j < QB; ++j) {
         int b = q0 + (j < nq ? j : 0);
         int64_t r = row_idx ? (int64_t)row_idx[b] : (int64_t)b;
         qrow[j] = reinterpret_cast<const uint4 *>(Q + r * ldq);
@@ -146,9 +149,9 @@ stream_lookup_kernel(const T *__restrict__ X, int64_t n_entries, int dim, const 
         for (int j = 0; j < nq; ++j)
             for (int c = tid; c < chunks; c += kStreamThreads) sq[j * chunks + c] = qrow[j][c];
 #pragma unroll
-        for (int j = 0; j < kQB; ++j) qrow[j] = sq + (j < nq ? j : 0) * chunks;
+        for (int j = 0; j < QB; ++j) qrow[j] = sq + (j < nq ? j : 0) * chunks;
     }
-    if (tid < kQB * kMaxK) {
+    if (tid < QB * kMaxK) {
         best_d[tid / kMaxK][tid % kMaxK] = __int_as_float(0x7F800000);
         best_i[tid / kMaxK][tid % kMaxK] = -1;
     }
@@ -157,48 +160,48 @@ stream_lookup_kernel(const T *__restrict__ X, int64_t n_entries, int dim, const 
     const int64_t r_begin = n_entries * blockIdx.x / parts;
     const int64_t r_end = n_entries * (blockIdx.x + 1) / parts;
 
-    for (int64_t r = r_begin; r < r_end; r += kRowsPerIter) {
-        float acc[kRowsPerIter][kQB];
+    for (int64_t r = r_begin; r < r_end; r += ROWS) {
+        float acc[ROWS][QB];
 #pragma unroll
-        for (int i = 0; i < kRowsPerIter; ++i)
+        for (int i = 0; i < ROWS; ++i)
 #pragma unroll
-            for (int j = 0; j < kQB; ++j) acc[i][j] = 0.f;
-        const uint4 *xrow[kRowsPerIter];
+            for (int j = 0; j < QB; ++j) acc[i][j] = 0.f;
+        const uint4 *xrow[ROWS];
 #pragma unroll
-        for (int i = 0; i < kRowsPerIter; ++i) {
+        for (int i = 0; i < ROWS; ++i) {
             int64_t rr = r + i < r_end ? r + i : r_end - 1;   // tail: re-read the last row, result ignored
             xrow[i] = reinterpret_cast<const uint4 *>(X + rr * dim);
         }
         for (int c = tid; c < chunks; c += kStreamThreads) {
-            uint4 xv[kRowsPerIter];
+            uint4 xv[ROWS];
 #pragma unroll
-            for (int i = 0; i < kRowsPerIter; ++i) xv[i] = ld_stream16(xrow[i] + c);
+            for (int i = 0; i < ROWS; ++i) xv[i] = ld_stream16(xrow[i] + c);
 #pragma unroll
-            for (int j = 0; j < kQB; ++j) {
+            for (int j = 0; j < QB; ++j) {
                 if (j < nq) {
                     uint4 qv = qrow[j][c];
 #pragma unroll
-                    for (int i = 0; i < kRowsPerIter; ++i) acc[i][j] = Elem<T>::sqdiff(qv, xv[i], acc[i][j]);
+                    for (int i = 0; i < ROWS; ++i) acc[i][j] = Elem<T>::sqdiff(qv, xv[i], acc[i][j]);
                 }
             }
         }
         // block reduction of the 16 partial sums
 #pragma unroll
-        for (int i = 0; i < kRowsPerIter; ++i)
+        for (int i = 0; i < ROWS; ++i)
 #pragma unroll
-            for (int j = 0; j < kQB; ++j) {
+            for (int j = 0; j < QB; ++j) {
                 float s = warp_sum(acc[i][j]);
-                if (lane == 0) red[warp][i * kQB + j] = s;
+                if (lane == 0) red[warp][i * QB + j] = s;
             }
         __syncthreads();
-        if (tid < kQB && tid < nq) {
+        if (tid < QB && tid < nq) {
             const int j = tid;
 #pragma unroll
-            for (int i = 0; i < kRowsPerIter; ++i) {
+            for (int i = 0; i < ROWS; ++i) {
                 if (r + i >= r_end) break;
                 float s = 0.f;
 #pragma unroll
-                for (int w = 0; w < kStreamWarps; ++w) s += red[w][i * kQB + j];
+                for (int w = 0; w < kStreamWarps; ++w) s += red[w][i * QB + j];
                 // insert (s, r+i) into the ascending list; rows arrive in ascending index, so "<" keeps the
                 // smaller index first among equal distances
                 if (s < best_d[j][k - 1]) {
@@ -251,35 +254,39 @@ fi_status_t launch_gather_rows(const void *src, int64_t ld_elems, const int32_t 
 fi_status_t launch_stream_lookup(const fi_cache *c, const void *queries, int64_t ld_elems, const int32_t *row_idx,
                                  int32_t batch_max, const int32_t *count_dev, int *parts_out, cudaStream_t stream) {
     const int k = c->cfg.k;
-    const int groups = (batch_max + kQB - 1) / kQB;
-    const int q_rows = batch_max < kQB ? batch_max : kQB;   // query rows a CTA actually holds
+    const bool single = batch_max == 1;
+    const int qb = single ? 1 : kQB, rows_per_iter = single ? kRowsPerIterSingle : kRowsPerIter;
+    const int groups = (batch_max + qb - 1) / qb;
+    const int q_rows = batch_max < qb ? batch_max : qb;   // query rows a CTA actually holds
     size_t q_bytes = (size_t)q_rows * c->cfg.dim * c->elem_size;
     int q_in_smem = q_bytes <= 160 * 1024;
     size_t dyn = q_in_smem ? q_bytes : 0;
-    const void *kern = c->cfg.dtype == FI_F32 ? (const void *)stream_lookup_kernel<float>
-                                              : (const void *)stream_lookup_kernel<uint16_t>;
+    const void *kern = c->cfg.dtype == FI_F32
+                           ? (single ? (const void *)stream_lookup_kernel<float, 1, kRowsPerIterSingle>
+                                     : (const void *)stream_lookup_kernel<float, kQB, kRowsPerIter>)
+                           : (single ? (const void *)stream_lookup_kernel<uint16_t, 1, kRowsPerIterSingle>
+                                     : (const void *)stream_lookup_kernel<uint16_t, kQB, kRowsPerIter>);
     if (dyn > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     int per_sm = 1;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kStreamThreads, dyn) != cudaSuccess || per_sm < 1)
         per_sm = 1;
-    // one wave of resident CTAs, but never more ranges than rows / 4 or than the scratch holds
+    // one wave of resident CTAs, but never more ranges than rows / rows per pass or than the scratch holds
     int parts = (per_sm * c->sm_count + groups - 1) / groups;
-    int64_t max_parts_rows = (c->size + kRowsPerIter - 1) / kRowsPerIter;
+    int64_t max_parts_rows = (c->size + rows_per_iter - 1) / rows_per_iter;
     if (parts > max_parts_rows) parts = (int)max_parts_rows;
     int64_t max_parts_scratch = (int64_t)(c->part_entries / ((size_t)batch_max * (size_t)k));
     if (parts > max_parts_scratch) parts = (int)max_parts_scratch;
     if (parts < 1) parts = 1;
     *parts_out = parts;
     dim3 grid((unsigned)parts, (unsigned)groups);
-    if (c->cfg.dtype == FI_F32) {
-        stream_lookup_kernel<float><<<grid, kStreamThreads, dyn, stream>>>((const float *)c->rows, c->size, c->cfg.dim, (const float *)queries,
-                                                    ld_elems, row_idx, batch_max, count_dev, k, parts, q_in_smem,
-                                                    c->part_score, c->part_idx);
-    } else {
-        stream_lookup_kernel<uint16_t><<<grid, kStreamThreads, dyn, stream>>>((const uint16_t *)c->rows, c->size, c->cfg.dim,
-                                                    (const uint16_t *)queries, ld_elems, row_idx, batch_max, count_dev, k,
-                                                    parts, q_in_smem, c->part_score, c->part_idx);
-    }
+    const void *rows = c->rows;
+    int64_t n = c->size;
+    int dim = c->cfg.dim, k_arg = k;
+    float *part_score = c->part_score;
+    int32_t *part_idx = c->part_idx;
+    void *args[] = {&rows, &n, &dim, &queries, &ld_elems, &row_idx, &batch_max, &count_dev, &k_arg, &parts, &q_in_smem,
+                    &part_score, &part_idx};
+    cudaLaunchKernel(kern, grid, dim3(kStreamThreads), args, dyn, stream);   // (a failed launch is reported below)
     count_launch();
     return check_launch("stream_lookup_kernel");
 }
