@@ -120,7 +120,7 @@ __global__ void gather_rows_kernel(const char *__restrict__ src, int64_t ld_byte
 // grid = (parts, ceil(batch_max / QB)); CTA (p, g) scans the p-th range of cache rows for queries QB*g..QB*g+QB-1 and
 // writes one sorted list of the k best (distance, index) pairs per query.  (QB, ROWS) = (4, 4), or (1, 8) for one request.
 template <typename T, int QB, int ROWS>
-__global__ void __launch_bounds__(kStreamThreads)
+__global__ void __launch_bounds__(kStreamThreads, QB == 1 ? 4 : 3)
 stream_lookup_kernel(const T *__restrict__ X, int64_t n_entries, int dim, const T *__restrict__ Q, int64_t ldq,
                      const int32_t *__restrict__ row_idx, int32_t batch_max, const int32_t *__restrict__ count_dev,
                      int k, int parts, int q_in_smem, float *__restrict__ part_score, int32_t *__restrict__ part_idx) {
