@@ -19,6 +19,7 @@ constexpr int kCertWords = 5;      // certificate block: uncertified, max score 
                                    // max ||c||^2 (float bits), uncertified and not repaired
 constexpr int kMaxPending = 16;    // inserts that may be in flight on a cache at once
 constexpr int kMaxDevices = 64;    // device ordinals the per-device set-up tables cover
+constexpr int kMinMapRows = 4;     // fewest rows a query tensor map is made over
 constexpr int kProfSlots = 256;    // look-ups whose distance-kernel time is kept
 
 // Candidates kept per query by the GEMM path before the exact re-ranking: k plus a margin of 3,

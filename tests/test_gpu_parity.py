@@ -95,6 +95,8 @@ def test_stream_path_large_dim_reads_queries_in_place():
     (5003, 200, 300, 5),       # 3 query tiles (last ragged), ragged N, K = 3 blocks + 8
     (40000, 64, 129, 10),      # one k-block, many row ranges, 2 query tiles
     (600, 1024, 5, 1),         # tiny batch, fewer 16-row blocks than CTAs
+    (3000, 1024, 2, 5),        # batches of 2 and 3 are copied into a four-row buffer in front of the GEMM
+    (700, 4096, 3, 1),
     (16, 8, 17, 5),            # a single 16-row block
     (3000, 4096, 64, 13),      # list length 16, deep K
     (2500, 136, 2200, 29),     # 18 query tiles (two groups), list length 32
