@@ -130,10 +130,12 @@ __device__ __forceinline__ bool certified(float d_k, float s_last, float qq, flo
 __device__ __forceinline__ bool pair_less(float s, int i, float t, int j) { return s < t || (s == t && i < j); }
 
 // One query, finished by all threads of a CTA together.
-// kLong: rows of at least kLongRowChunks 16-byte chunks take the exact distances by slices of the row (below)
+// kLong: rows of at least kLongRowChunks 16-byte chunks take the exact distances by slices of the row (below);
+// kLong == 2: the same for candidate lists of at most four entries (k = 1), four candidates and two blocks of the row
+// per step instead of eight candidates and one, so that as many loads are in flight
 constexpr int kLongRowChunks = 1024;
 
-template <typename T, bool kLong>
+template <typename T, int kLong>
 __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int b, int parts, int list_len) {
     __shared__ float cand_s[kMaxK];
     __shared__ float cand_d[kMaxK];
@@ -291,7 +293,8 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
     // this architecture, two elements per instruction, were measured here too: slower, and 16 more registers.)
     // The partial sums are added in a fixed order (lanes by shuffle tree, then warps 0..7), so reruns are bit-identical.
     if (p.refine) {
-        constexpr int kGroup = 8;   // candidates per pass over the query
+        constexpr int kGroup = kLong == 2 ? 4 : 8;   // candidates per pass over the query
+        constexpr int kBlocks = kLong == 2 ? 2 : 1;  // blocks of the row per step
         __shared__ float part[kFinWarps][kGroup + 1];
         const int64_t qr = p.row_idx ? (int64_t)p.row_idx[b] : (int64_t)b;
         const uint4 *q4 = reinterpret_cast<const uint4 *>(reinterpret_cast<const T *>(p.Q) + qr * p.ldq);
@@ -344,16 +347,28 @@ __device__ __forceinline__ void finalize_query_cta(const FinalizeParams &p, int 
 #pragma unroll
                 for (int u = 0; u < kGroup; ++u) a[u] = 0.f;
                 const bool with_norm = j0 == 0;   // ||q||^2 for the certificate rides along with the first pass
-                for (int c = warp * 32 + lane; c < chunks; c += kFinWarps * 32) {
-                    const uint4 qv = ld16(q4 + c);
-                    uint4 xv[kGroup];
+                for (int c = warp * 32 + lane; c < chunks; c += kBlocks * kFinWarps * 32) {
+                    uint4 qv[kBlocks], xv[kBlocks][kGroup];
 #pragma unroll
-                    for (int u = 0; u < kGroup; ++u)
-                        if (u < nj) xv[u] = ld16(x[u] + c);
+                    for (int s2 = 0; s2 < kBlocks; ++s2) {
+                        const int cc = c + s2 * kFinWarps * 32;
+                        if (cc < chunks) {
+                            qv[s2] = ld16(q4 + cc);
 #pragma unroll
-                    for (int u = 0; u < kGroup; ++u)
-                        if (u < nj) a[u] = sqdiff16<T>(qv, xv[u], a[u]);
-                    if (with_norm) nq = sqnorm16<T>(qv, nq);
+                            for (int u = 0; u < kGroup; ++u)
+                                if (u < nj) xv[s2][u] = ld16(x[u] + cc);
+                        }
+                    }
+                    // (the sums grow block after block, as with one block per step)
+#pragma unroll
+                    for (int s2 = 0; s2 < kBlocks; ++s2) {
+                        if (c + s2 * kFinWarps * 32 < chunks) {
+#pragma unroll
+                            for (int u = 0; u < kGroup; ++u)
+                                if (u < nj) a[u] = sqdiff16<T>(qv[s2], xv[s2][u], a[u]);
+                            if (with_norm) nq = sqnorm16<T>(qv[s2], nq);
+                        }
+                    }
                 }
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) {
@@ -708,7 +723,7 @@ __global__ void __launch_bounds__(kFinThreads) finalize_kernel(FinalizeParams p)
     if (b >= count) return;
     const int parts = p.plan ? p.plan->lists : p.parts;
     const int list_len = p.plan ? p.plan->list_len : p.list_len;
-    finalize_query_cta<T, false>(p, b, parts, list_len);
+    finalize_query_cta<T, 0>(p, b, parts, list_len);
 }
 
 // The same for long rows (16 KiB and more): the slice-wise exact distances hold eight candidates' partial sums per
@@ -720,7 +735,18 @@ __global__ void __launch_bounds__(kFinThreads, 4) finalize_long_kernel(FinalizeP
     if (b >= count) return;
     const int parts = p.plan ? p.plan->lists : p.parts;
     const int list_len = p.plan ? p.plan->list_len : p.list_len;
-    finalize_query_cta<T, true>(p, b, parts, list_len);
+    finalize_query_cta<T, 1>(p, b, parts, list_len);
+}
+
+// Long rows under lists of at most four entries (k = 1: the latency regime).
+template <typename T>
+__global__ void __launch_bounds__(kFinThreads, 4) finalize_long_few_kernel(FinalizeParams p) {
+    const int count = p.count_dev ? min(*p.count_dev, p.batch_max) : p.batch_max;
+    const int b = blockIdx.x;
+    if (b >= count) return;
+    const int parts = p.plan ? p.plan->lists : p.parts;
+    const int list_len = p.plan ? p.plan->list_len : p.list_len;
+    finalize_query_cta<T, 2>(p, b, parts, list_len);
 }
 
 // Short rows.  Large batches (k-means assignment, threshold calibration) whose candidate entries fit a warp's
@@ -743,7 +769,7 @@ __global__ void __launch_bounds__(kFinThreads) finalize_rows_kernel(FinalizePara
         const int b = blockIdx.x * kFinWarps + warp;
         if (b < count) finalize_query_warp<T>(p, b, parts, list_len, sort_d[warp], sort_i[warp], sort_lab[warp], sort_w[warp]);
     } else if ((int)blockIdx.x < count) {
-        finalize_query_cta<T, false>(p, blockIdx.x, parts, list_len);
+        finalize_query_cta<T, 0>(p, blockIdx.x, parts, list_len);
     }
 }
 
@@ -981,13 +1007,16 @@ fi_status_t launch_finalize(const fi_cache *c, const FinalizeArgs &a, cudaStream
     // (the plain kernel needs fewer registers, so more of its CTAs are resident)
     const bool short_rows = (size_t)c->cfg.dim * c->elem_size <= 8192 && a.batch_max >= kWarpModeMinBatch;
     const int grid = a.batch_max;
+    const bool few = gemm_list_len(c->cfg.k) <= 4;   // the tensor-core path's lists for k = 1
     const bool long_rows = a.refine && (size_t)c->cfg.dim * c->elem_size >= (size_t)kLongRowChunks * 16;
     if (c->cfg.dtype == FI_F32) {
         if (short_rows) finalize_rows_kernel<float><<<grid, kFinThreads, 0, stream>>>(p);
+        else if (long_rows && few) finalize_long_few_kernel<float><<<grid, kFinThreads, 0, stream>>>(p);
         else if (long_rows) finalize_long_kernel<float><<<grid, kFinThreads, 0, stream>>>(p);
         else finalize_kernel<float><<<grid, kFinThreads, 0, stream>>>(p);
     } else {
         if (short_rows) finalize_rows_kernel<uint16_t><<<grid, kFinThreads, 0, stream>>>(p);
+        else if (long_rows && few) finalize_long_few_kernel<uint16_t><<<grid, kFinThreads, 0, stream>>>(p);
         else if (long_rows) finalize_long_kernel<uint16_t><<<grid, kFinThreads, 0, stream>>>(p);
         else finalize_kernel<uint16_t><<<grid, kFinThreads, 0, stream>>>(p);
     }
