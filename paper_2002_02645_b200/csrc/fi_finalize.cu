@@ -751,9 +751,9 @@ __global__ void __launch_bounds__(kFinThreads, 4) finalize_long_few_kernel(Final
 
 // Short rows.  Large batches (k-means assignment, threshold calibration) whose candidate entries fit a warp's
 // registers are finished one query per warp, kFinWarps consecutive queries per CTA: a CTA per query would spend its time
-// on barriers and on CTA launches (40,000 queries: 0.26 -> 0.09 ms).  Smaller batches keep the CTA per query, whose
-// latency is shorter.  The grid always has one CTA per slot of the batch; the CTAs left without work return at once.
-constexpr int kWarpModeMinBatch = 8192;
+// on barriers and on CTA launches (40,000 queries: 0.26 -> 0.09 ms; 1,282 to 4,096 queries of 256 to 2,048 values: a
+// four-stage cascade 1.513 -> 1.499 ms).  Batches below 1,024 keep the CTA per query, whose latency is shorter.  The grid always has one CTA per slot of the batch; the CTAs left without work return at once.
+constexpr int kWarpModeMinBatch = 1024;
 
 template <typename T>
 __global__ void __launch_bounds__(kFinThreads) finalize_rows_kernel(FinalizeParams p) {
