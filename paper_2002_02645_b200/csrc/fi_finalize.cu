@@ -756,7 +756,7 @@ __global__ void __launch_bounds__(kFinThreads, 4) finalize_long_few_kernel(Final
 constexpr int kWarpModeMinBatch = 1024;
 
 template <typename T>
-__global__ void __launch_bounds__(kFinThreads) finalize_rows_kernel(FinalizeParams p) {
+__global__ void __launch_bounds__(kFinThreads, 4) finalize_rows_kernel(FinalizeParams p) {
     __shared__ float sort_d[kFinWarps][kMaxK];
     __shared__ int32_t sort_i[kFinWarps][kMaxK];
     __shared__ int32_t sort_lab[kFinWarps][kMaxK];

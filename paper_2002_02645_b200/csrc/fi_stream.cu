@@ -109,6 +109,16 @@ __global__ void gather_rows_kernel(const char *__restrict__ src, int64_t ld_byte
                                    int row_bytes) {
     int count = count_dev ? min(*count_dev, batch_max) : batch_max;
     int chunks = row_bytes / 16;
+    if (chunks <= 256) {
+        // short rows: a row per warp (a CTA of 256 threads would leave most of them without a chunk)
+        const int warps = blockDim.x >> 5, lane = threadIdx.x & 31;
+        for (int b = blockIdx.x * warps + (threadIdx.x >> 5); b < count; b += gridDim.x * warps) {
+            const uint4 *s = reinterpret_cast<const uint4 *>(src + (int64_t)row_idx[b] * ld_bytes);
+            uint4 *d = reinterpret_cast<uint4 *>(dst + (int64_t)b * row_bytes);
+            for (int c = lane; c < chunks; c += 32) d[c] = ld_stream16(s + c);
+        }
+        return;
+    }
     for (int b = blockIdx.x; b < count; b += gridDim.x) {
         const uint4 *s = reinterpret_cast<const uint4 *>(src + (int64_t)row_idx[b] * ld_bytes);
         uint4 *d = reinterpret_cast<uint4 *>(dst + (int64_t)b * row_bytes);
@@ -245,7 +255,10 @@ fi_status_t launch_row_norms(const void *rows, int dtype, int64_t n, int dim, fl
 fi_status_t launch_gather_rows(const void *src, int64_t ld_elems, const int32_t *row_idx, int32_t batch_max,
                                const int32_t *count_dev, void *dst, int dim, size_t elem_size, cudaStream_t stream) {
     if (batch_max <= 0) return FI_OK;
-    gather_rows_kernel<<<batch_max, 256, 0, stream>>>((const char *)src, ld_elems * (int64_t)elem_size, row_idx, count_dev,
+    // (rows of up to 4 KiB go a row per warp, eight rows per CTA)
+    const int row_chunks = (int)(dim * elem_size / 16);
+    const int grid = row_chunks <= 256 ? (batch_max + 7) / 8 : batch_max;
+    gather_rows_kernel<<<grid, 256, 0, stream>>>((const char *)src, ld_elems * (int64_t)elem_size, row_idx, count_dev,
                                                       batch_max, (char *)dst, (int)(dim * elem_size));
     count_launch();
     return check_launch("gather_rows_kernel");
